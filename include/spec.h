@@ -1,0 +1,180 @@
+/*
+ * spec.h -- C ABI of the B200 (sm_100a) lookahead-importance library.
+ *
+ * The library implements the data-parallel hot path of draft-based approximate
+ * inference: SpecKV's lookahead importance scoring, pooling, top-C_max selection
+ * and K/V compaction (Algorithm 1, lines 8-15; Eq. 1), and the SpecPC keep set
+ * built on the same scores (Algorithm 2, lines 7-10).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library
+ *     never allocates, frees or retains them.  Scratch memory is passed in as
+ *     `workspace` (size from spec_workspace_bytes); its contents are undefined
+ *     on entry and on return.
+ *   - Work is enqueued asynchronously on `stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream).  The int32 return value is a
+ *     spec_status: argument errors are detected on the host before anything is
+ *     launched; launch failures map to SPEC_ERR_CUDA.  Nothing throws, aborts
+ *     or prints; spec_last_error() gives a human-readable reason.
+ *   - `status_word` (optional device int32, caller zeroes it) receives a
+ *     negative spec_status if a kernel gave up on a bounded wait; read it after
+ *     synchronising the stream.  The outputs of that call are then undefined.
+ *   - There is no CPU fallback: on a device that is not compute capability
+ *     10.x every compute entry point returns SPEC_ERR_UNSUPPORTED.
+ *   - Calls that share a workspace or an output buffer must not overlap on the
+ *     GPU; calls on one stream are ordered and need no host synchronisation
+ *     between them.
+ *
+ * Notation (the paper's): n_in prompt length, R = n_window + n_lookahead query
+ * rows per query head, G = n_q_heads / n_kv_heads, M = G*R query rows that
+ * share one KV head, d = head_dim, L = n_layers, T = total_tokens.
+ */
+#ifndef SPEC_H_
+#define SPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPEC_OK = 0,
+  SPEC_ERR_BAD_ARG = -1,        /* NULL pointer, size out of range, inconsistent arguments */
+  SPEC_ERR_ALIGNMENT = -2,      /* pointer or stride not 16-byte aligned */
+  SPEC_ERR_UNSUPPORTED = -3,    /* shape outside the implemented range, or not an sm_100 device */
+  SPEC_ERR_WORKSPACE = -4,      /* workspace NULL or smaller than spec_workspace_bytes() */
+  SPEC_ERR_CUDA = -5,           /* a CUDA runtime / driver call failed */
+  SPEC_ERR_TIMEOUT = -6,        /* device side: a bounded wait expired (status_word only) */
+  SPEC_ERR_NOT_IMPLEMENTED = -7
+} spec_status;
+
+/* Reduction over query rows (spec_score) or over layers and heads (specpc_token_select). */
+typedef enum {
+  SPEC_REDUCE_SUM = 0,          /* Eq. 1 up to the constant 1/rows */
+  SPEC_REDUCE_MAX = 1           /* Algorithm 1 line 9 / Algorithm 2 line 7 (MaxReduce) */
+} spec_reduce;
+
+typedef enum {
+  SPEC_POOL_MAX = 0,            /* hyper-parameter table: SpecKV pools with Max, k = 7 */
+  SPEC_POOL_AVG = 1             /* Algorithm 1 line 10 / Algorithm 2 line 8 as printed (AvgPool1D) */
+} spec_pool;
+
+/*
+ * Problem geometry shared by all calls.
+ *
+ * Keys and values live on a packed token axis of extent total_tokens; sequence s
+ * owns tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (n_s of them; cu_seqlens is a
+ * DEVICE array of n_seq+1 non-decreasing int32 with cu_seqlens[n_seq] <=
+ * total_tokens).  cu_seqlens == NULL means one sequence covering tokens
+ * [0, n_in).  Element (layer, kv_head, token, c) of K is at
+ *   k + layer*k_stride_layer + kv_head*k_stride_head + token*k_stride_token + c
+ * (strides in elements, bf16; the head_dim axis is contiguous); V likewise.
+ * K/V base pointers and strides*2 bytes must be multiples of 16 bytes.
+ */
+typedef struct {
+  int32_t n_seq;                /* >= 1 (<= 1024) */
+  const int32_t* cu_seqlens;    /* device [n_seq+1] or NULL */
+  int32_t n_in;                 /* used only when cu_seqlens == NULL */
+  int32_t total_tokens;         /* T */
+  int32_t n_layers, n_q_heads, n_kv_heads, head_dim;   /* head_dim in {64, 128}; n_q_heads % n_kv_heads == 0 */
+  int32_t n_lookahead, n_window;                        /* R >= 1; n_lookahead may be 0 (SnapKV special case) */
+  float softmax_scale;          /* > 0; Eq. 1 uses 1/sqrt(head_dim) */
+  int64_t k_stride_layer, k_stride_head, k_stride_token;
+  int64_t v_stride_layer, v_stride_head, v_stride_token;
+} spec_problem;
+
+/* Bytes of scratch that any of the calls below may need for this problem (0 on a bad problem). */
+size_t spec_workspace_bytes(const spec_problem* problem);
+
+/* Reason of the calling thread's last non-OK return (static storage, never NULL). */
+const char* spec_last_error(void);
+
+/*
+ * Importance scores -- Eq. 1; Algorithm 1 lines 8-9 (CrossAttention of the window
+ * and lookahead queries against the prompt keys, reduced over query rows).
+ *
+ * For every (sequence, layer, KV head) the M = G*R query rows of the GQA group are
+ * scored against the sequence's keys with a per-row softmax of
+ * softmax_scale * <q, k>, and the probabilities are reduced over the M rows:
+ *   SPEC_REDUCE_SUM: scores[j] = sum_i w_i p_i[j]     SPEC_REDUCE_MAX: max_i w_i p_i[j]
+ * The M x n_s probability matrix is never written to memory.
+ *
+ *  q           [n_seq, n_layers, n_q_heads, R, head_dim] bf16, contiguous, 16-byte aligned; rows are
+ *              the n_window last prompt tokens in prompt order, then the lookahead tokens
+ *              (Algorithm 1 line 8, "[X_m: ; Y]")
+ *  k           bf16, see spec_problem
+ *  row_weight  optional device float[R], w >= 0 (Algorithm 2 lines 4-6); NULL = all ones
+ *  causal_window  0: every row sees every key it is given.  1: window row r only sees keys up to
+ *              its own prompt position n_s - n_window + r.
+ *  scores_out  [n_layers, n_kv_heads, T] fp32; only tokens covered by cu_seqlens are written
+ * Limits: M*head_dim <= 81920 (e.g. M <= 640 at head_dim 128); else SPEC_ERR_UNSUPPORTED.
+ */
+int32_t spec_score(const spec_problem* problem, const void* q, const void* k, const float* row_weight,
+                   int32_t reduce, int32_t causal_window, float* scores_out, void* workspace,
+                   size_t workspace_bytes, int32_t* status_word, void* stream);
+
+/*
+ * Pooling + top-C_max selection -- Algorithm 1 lines 10 and 13.
+ *
+ * Per (sequence, layer, KV head), with e = n_s - min(n_forced_tail, n_s) eligible positions
+ * [0, e): pooled[j] = pool over scores[j - pool_k/2 .. j - pool_k/2 + pool_k - 1] clipped to
+ * [0, e) (stride 1; AVG divides by pool_k), the min(c_max - forced, e) positions with the largest
+ * pooled value are kept (equal values: the lower position wins), and the forced tail [e, n_s) is
+ * always kept (Algorithm 1 line 13: the last n_window KV pairs).  n_forced_tail = 0 selects the
+ * plain top-c_max over all n_s positions.
+ *
+ *  scores     [n_layers, n_kv_heads, T] fp32, non-negative
+ *  idx_out    [n_seq, n_layers, n_kv_heads, c_max] int32, ascending sequence-local positions,
+ *             padded with -1 when fewer than c_max positions exist
+ *  count_out  optional [n_seq, n_layers, n_kv_heads] int32 number of valid entries
+ * Requires 1 <= pool_k <= 255, 0 <= n_forced_tail <= c_max, c_max >= 1.
+ */
+int32_t spec_pool_topk(const spec_problem* problem, const float* scores, int32_t pool, int32_t pool_k,
+                       int32_t c_max, int32_t n_forced_tail, int32_t* idx_out, int32_t* count_out,
+                       void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
+
+/*
+ * K/V compaction -- Algorithm 1 line 15 (cache <- K[i_cache], V[i_cache]).
+ *
+ * Row c of the compacted cache of (sequence s, layer, KV head) is source token
+ * cu_seqlens[s] + idx[s, layer, head, c]; rows whose idx is -1 are zero-filled.  Rows are copied
+ * bit-exactly.  v / v_out may both be NULL to gather K only.
+ *
+ *  block_table == NULL: k_out, v_out are [n_seq, n_layers, n_kv_heads, c_max, head_dim] bf16.
+ *  block_table != NULL: k_out, v_out are page pools [n_layers, n_pages, n_kv_heads, page_size,
+ *             head_dim]; slot c of sequence s goes to page block_table[s, c / page_size] (device
+ *             int32 [n_seq, ceil(c_max / page_size)], assigned by the caller, each id in
+ *             [0, n_pages)), row c % page_size.  Ids out of range are skipped and reported as
+ *             SPEC_ERR_BAD_ARG in status_word.
+ */
+int32_t spec_compact_kv(const spec_problem* problem, const void* k, const void* v, const int32_t* idx,
+                        int32_t c_max, void* k_out, void* v_out, const int32_t* block_table,
+                        int32_t page_size, int32_t n_pages, int32_t* status_word, void* stream);
+
+/*
+ * SpecPC keep set -- Algorithm 2 lines 7-10.
+ *
+ * Per sequence: token score t[j] = reduce over all layers and KV heads of scores[l, h, j]
+ * (`layer_head_reduce`; skip the first l_skip layers by offsetting `scores` and shrinking
+ * problem->n_layers), pooled as in spec_pool_topk, top-c_max positions selected, every selected
+ * position widened to [i - n_neighbor, i + n_neighbor] inside the eligible range, the forced tail
+ * (the always-kept window) added, and the distinct positions written in ascending order.
+ *
+ *  scores      [n_layers, n_kv_heads, T] fp32 from spec_score on the draft model's Q/K
+ *  keep_out    [n_seq, keep_capacity] int32, ascending, padded with -1
+ *  n_keep_out  [n_seq] int32
+ * keep_capacity must be >= min(max_len, c_max*(2*n_neighbor+1) + n_forced_tail) where max_len is
+ * n_in (cu_seqlens == NULL) or total_tokens; else SPEC_ERR_BAD_ARG.
+ */
+int32_t specpc_token_select(const spec_problem* problem, const float* scores, int32_t layer_head_reduce,
+                            int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,
+                            int32_t n_forced_tail, int32_t* keep_out, int32_t keep_capacity,
+                            int32_t* n_keep_out, void* workspace, size_t workspace_bytes,
+                            int32_t* status_word, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPEC_H_ */

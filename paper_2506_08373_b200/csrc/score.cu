@@ -1,0 +1,660 @@
+// Lookahead importance scoring (Eq. 1; Algorithm 1 lines 8-9) on tcgen05 tensor cores.
+//
+// score[j] = reduce_i softmax_j(scale * q_i . k_j) over the M = G*R query rows that share a
+// KV head.  The M x n probability matrix never leaves the SM:
+//   pass 1   S = Q K^T per 128-key tile (query rows on TMEM lanes): running row max and
+//            sum-exp, kept per thread, written per (CTA, unit) segment;
+//   merge    combines the segments' statistics into one constant per row,
+//            c_i = log2e*scale*max_i + log2 Z_i - log2 w_i;
+//   pass 2   S^T = K Q^T per tile (keys on TMEM lanes, query rows on columns):
+//            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one store per key.
+// Both passes are persistent, warp-specialised kernels: warp 0 feeds K tiles (and the unit's Q)
+// with TMA into a shared-memory ring, warp 1 issues tcgen05.mma into double-buffered TMEM, warps
+// 2-5 drain TMEM with tcgen05.ld and do the exponentials.  The global key-tile space
+// (layer, KV head, sequence, tile) is cut into equal contiguous ranges, one per CTA.
+//
+// Every wait on an mbarrier is bounded in time; on expiry the CTA reports SPEC_ERR_TIMEOUT
+// through the status word, lets its copies land, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace spec {
+
+constexpr int kThreads = 192;
+constexpr int kTileKeys = 128;
+constexpr int kMaxStages = 8;
+constexpr int kMaxMTiles = 10;
+constexpr int kNumBars = 2 * kMaxStages + 2 + 8;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct ScoreParams {
+  const int32_t* cu;
+  const float* row_weight;
+  float* partial;       // [n_units + n_ctas][M][2]  (max in log2 domain, sum-exp)
+  float* rowc;          // [n_seq*L*Hq*R]  minus the per-row constant
+  float* scores;        // [L, Hkv, T]
+  int32_t* status;
+  long long T;
+  int n_in, n_seq, L, Hq, Hkv, G, R, M, M_pad, d;
+  int n_stages, n_chunks, cw, cw_last;
+  int reduce;
+  float a;              // softmax_scale * log2(e)
+  uint32_t q_bytes, stage_bytes;
+};
+
+// ------------------------------------------------------------------ PTX wrappers ------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when another role has given up or the time limit passed.
+__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t addr = smem_u32(bar);
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int x, int y, int z, int w, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulation, issued by one thread.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+// Completes all earlier tcgen05.ld of this thread; the registers are tied to the wait so that
+// no use of them can be scheduled above it.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor: K-major operand, rows of 64 bf16 (128 bytes) with the
+// 128-byte swizzle TMA writes; 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                 // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ------------------------------------------------------------- work decomposition -----
+
+struct Seg {
+  int unit;        // ordinal (layer*Hkv + head)*n_seq + seq
+  int s, l, h;
+  int begin, n;    // token range of the sequence
+  int t0, nt;      // first key tile of the unit handled here, number of tiles
+};
+
+struct SegIter {
+  long long g, g_end;
+  int TT;
+};
+
+// Tile-count prefix over sequences, tp[0..n_seq].
+__device__ void build_tile_prefix(const ScoreParams& p, int* tp) {
+  int acc = 0;
+  tp[0] = 0;
+  for (int s = 0; s < p.n_seq; ++s) {
+    int b, n;
+    seq_range(p.cu, p.n_in, s, b, n);
+    acc += (n + kTileKeys - 1) / kTileKeys;
+    tp[s + 1] = acc;
+  }
+}
+
+__device__ __forceinline__ SegIter seg_begin(const ScoreParams& p, const int* tp, int n_ctas, int cta) {
+  SegIter it;
+  it.TT = tp[p.n_seq];
+  const long long N = (long long)p.L * p.Hkv * it.TT;
+  const long long P = (N + n_ctas - 1) / n_ctas;
+  it.g = P * cta;
+  it.g_end = it.g + P < N ? it.g + P : N;
+  return it;
+}
+
+__device__ bool seg_next(SegIter& it, const ScoreParams& p, const int* tp, Seg& sg) {
+  if (it.g >= it.g_end) return false;
+  const int lh = (int)(it.g / it.TT);
+  const int rem = (int)(it.g % it.TT);
+  int lo = 0, hi = p.n_seq;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tp[mid] <= rem) lo = mid; else hi = mid;
+  }
+  sg.s = lo;
+  sg.l = lh / p.Hkv;
+  sg.h = lh % p.Hkv;
+  sg.unit = lh * p.n_seq + lo;
+  sg.t0 = rem - tp[lo];
+  const long long left = it.g_end - it.g;
+  const int in_unit = tp[lo + 1] - rem;
+  sg.nt = left < in_unit ? (int)left : in_unit;
+  seq_range(p.cu, p.n_in, lo, sg.begin, sg.n);
+  it.g += sg.nt;
+  return true;
+}
+
+// ------------------------------------------------------------------ epilogue math -----
+
+// Pass 1: fold 32 logits of one row into the running (max, sum-exp), log2 domain.
+template <bool MASKED>
+__device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid, float a, float& m, float& z) {
+  float gm = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const float v = __uint_as_float(r[i]);
+    if (!MASKED || i < valid) gm = fmaxf(gm, v);
+  }
+  const float mn = fmaxf(m, gm * a);
+  if (mn == -INFINITY) return;
+  const float neg = -mn;
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    float e0 = ex2(fmaf(__uint_as_float(r[i + 0]), a, neg));
+    float e1 = ex2(fmaf(__uint_as_float(r[i + 1]), a, neg));
+    float e2 = ex2(fmaf(__uint_as_float(r[i + 2]), a, neg));
+    float e3 = ex2(fmaf(__uint_as_float(r[i + 3]), a, neg));
+    if (MASKED) {
+      if (i + 0 >= valid) e0 = 0.f;
+      if (i + 1 >= valid) e1 = 0.f;
+      if (i + 2 >= valid) e2 = 0.f;
+      if (i + 3 >= valid) e3 = 0.f;
+    }
+    s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+  }
+  z = z * ex2(m - mn) + ((s0 + s1) + (s2 + s3));
+  m = mn;
+}
+
+// Pass 2: probabilities of 32 query rows for this thread's key, reduced into acc[4].
+template <bool MAXRED>
+__device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const float* __restrict__ negc, float a, float (&acc)[4]) {
+  const float4* c4 = reinterpret_cast<const float4*>(negc);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float4 c = c4[i];
+    const float p0 = ex2(fmaf(__uint_as_float(r[4 * i + 0]), a, c.x));
+    const float p1 = ex2(fmaf(__uint_as_float(r[4 * i + 1]), a, c.y));
+    const float p2 = ex2(fmaf(__uint_as_float(r[4 * i + 2]), a, c.z));
+    const float p3 = ex2(fmaf(__uint_as_float(r[4 * i + 3]), a, c.w));
+    if (MAXRED) {
+      acc[0] = fmaxf(acc[0], p0); acc[1] = fmaxf(acc[1], p1); acc[2] = fmaxf(acc[2], p2); acc[3] = fmaxf(acc[3], p3);
+    } else {
+      acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ the kernel --------
+
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  constexpr int BUFCOLS = PASS == 1 ? 128 : 256;
+  constexpr int NBUF = 512 / BUFCOLS;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint8_t* k_sm = smem;
+  uint8_t* q_sm = smem + (size_t)p.n_stages * p.stage_bytes;
+  float* c_sm = reinterpret_cast<float*>(q_sm + p.q_bytes);
+  int* tp = reinterpret_cast<int*>(c_sm + p.M_pad);
+  uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(tp + p.n_seq + 1) + 7) & ~(uintptr_t)7);
+  uint64_t* k_full = bars;
+  uint64_t* k_empty = bars + kMaxStages;
+  uint64_t* q_full = bars + 2 * kMaxStages;
+  uint64_t* q_empty = q_full + 1;
+  uint64_t* t_full = q_full + 2;
+  uint64_t* t_empty = t_full + 4;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  if ((smem_u32(smem) & 1023u) != 0) {      // the swizzled tiles need 1024-byte alignment
+    if (tid == 0) report(p.status, SPEC_ERR_ALIGNMENT);
+    return;
+  }
+  if (tid == 0) {
+    *abort_flag = 0;
+    build_tile_prefix(p, tp);
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+  }
+  if (tid == 32) {
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+    mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_kh = p.d / 64;                               // 64-element halves of the contraction
+  const uint32_t q_half_bytes = (uint32_t)p.M_pad * 128u;
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer ----
+    if (lane == 0) {
+      SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
+      Seg sg;
+      uint32_t kit = 0, nseg = 0;
+      bool ok = true;
+      while (ok && seg_next(it, p, tp, sg)) {
+        if (nseg > 0) ok = mbar_wait(q_empty, (nseg - 1) & 1, abort_flag);   // previous unit's MMAs retired
+        if (!ok) break;
+        ++nseg;
+        mbar_expect_tx(q_full, p.q_bytes);
+        const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
+        for (int kh = 0; kh < n_kh; ++kh)
+          for (int rb = 0; rb < p.M_pad / 128; ++rb)
+            tma_load_2d(q_sm + kh * q_half_bytes + rb * (128 * 128), &tm_q, kh * 64, qrow0 + rb * 128, q_full);
+        for (int t = 0; t < sg.nt; ++t, ++kit) {
+          const int stage = kit % p.n_stages;
+          const uint32_t par = (kit / p.n_stages) & 1;
+          ok = mbar_wait(&k_empty[stage], par ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(&k_full[stage], p.stage_bytes);
+          uint8_t* dst = k_sm + (size_t)stage * p.stage_bytes;
+          const int row = sg.begin + (sg.t0 + t) * kTileKeys;
+          for (int kh = 0; kh < n_kh; ++kh)
+            tma_load_4d(dst + kh * (128 * 128), &tm_k, kh * 64, row, sg.h, sg.l, &k_full[stage]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer ------
+    if (lane == 0) {
+      SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
+      Seg sg;
+      uint32_t kit = 0, bit = 0, nseg = 0;
+      bool ok = true;
+      const uint32_t idesc_full = make_idesc(PASS == 1 ? 128 : p.cw);
+      const uint32_t idesc_last = make_idesc(PASS == 1 ? 128 : p.cw_last);
+      const int n_sub = PASS == 1 ? p.M_pad / 128 : p.n_chunks;
+      const uint32_t q_base = smem_u32(q_sm);
+      while (ok && seg_next(it, p, tp, sg)) {
+        ok = mbar_wait(q_full, nseg & 1, abort_flag);
+        if (!ok) break;
+        ++nseg;
+        tc_fence_after();
+        for (int t = 0; t < sg.nt && ok; ++t, ++kit) {
+          const int stage = kit % p.n_stages;
+          ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_base = smem_u32(k_sm + (size_t)stage * p.stage_bytes);
+          for (int sub = 0; sub < n_sub; ++sub, ++bit) {
+            const int buf = bit % NBUF;
+            ok = mbar_wait(&t_empty[buf], ((bit / NBUF) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
+            const uint32_t q_off = PASS == 1 ? sub * (128 * 128) : sub * p.cw * 128;
+            const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
+            for (int kh = 0; kh < n_kh; ++kh) {
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t qd = make_desc(q_base + kh * q_half_bytes + q_off + ks * 32);
+                const uint64_t kd = make_desc(k_base + kh * (128 * 128) + ks * 32);
+                if (PASS == 1) tc_mma(d_tmem, qd, kd, idesc, (kh | ks) != 0);
+                else           tc_mma(d_tmem, kd, qd, idesc, (kh | ks) != 0);
+              }
+            }
+            tc_commit(&t_full[buf]);
+          }
+          if (ok) tc_commit(&k_empty[stage]);      // stage reusable once these MMAs retire
+        }
+        if (ok) tc_commit(q_empty);
+      }
+    }
+  } else {
+    // ------------------------------------------------ epilogue --------
+    const int quarter = warp & 3;                          // TMEM lane quarter this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    const int et = tid - 64;                               // 0..127 among epilogue threads
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
+    Seg sg;
+    uint32_t bit = 0;
+    bool ok = true;
+    uint32_t ra[32], rb[32];
+    if (PASS == 1) {
+      const int n_mt = p.M_pad / 128;
+      float mrun[kMaxMTiles], zrun[kMaxMTiles];
+      while (ok && seg_next(it, p, tp, sg)) {
+#pragma unroll
+        for (int i = 0; i < kMaxMTiles; ++i) { mrun[i] = -INFINITY; zrun[i] = 0.f; }
+        for (int t = 0; t < sg.nt && ok; ++t) {
+          const int nv = min(kTileKeys, sg.n - (sg.t0 + t) * kTileKeys);
+          for (int mt = 0; mt < n_mt; ++mt, ++bit) {
+            const int buf = bit % NBUF;
+            ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = lane_base + buf * BUFCOLS;
+            float m = mrun[mt], z = zrun[mt];
+            tmem_ld32(taddr, ra);
+            tmem_ld_wait(ra);
+            tmem_ld32(taddr + 32, rb);
+            if (nv >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nv, p.a, m, z);
+            tmem_ld_wait(rb);
+            tmem_ld32(taddr + 64, ra);
+            if (nv >= 64) stats_update<false>(rb, 32, p.a, m, z); else if (nv > 32) stats_update<true>(rb, nv - 32, p.a, m, z);
+            tmem_ld_wait(ra);
+            tmem_ld32(taddr + 96, rb);
+            if (nv >= 96) stats_update<false>(ra, 32, p.a, m, z); else if (nv > 64) stats_update<true>(ra, nv - 64, p.a, m, z);
+            tmem_ld_wait(rb);
+            if (nv >= 128) stats_update<false>(rb, 32, p.a, m, z); else if (nv > 96) stats_update<true>(rb, nv - 96, p.a, m, z);
+            mrun[mt] = m;
+            zrun[mt] = z;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&t_empty[buf]);
+          }
+        }
+        if (ok) {
+          float* dst = p.partial + (size_t)(sg.unit + blockIdx.x) * p.M * 2;
+          for (int mt = 0; mt < n_mt; ++mt) {
+            const int row = mt * 128 + row_in_tile;
+            if (row < p.M) {
+              dst[row * 2 + 0] = mrun[mt];
+              dst[row * 2 + 1] = zrun[mt];
+            }
+          }
+        }
+      }
+    } else {
+      while (ok && seg_next(it, p, tp, sg)) {
+        const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
+        asm volatile("bar.sync 1, 128;" ::: "memory");          // previous unit's constants no longer read
+        for (int i = et; i < p.M_pad; i += 128) c_sm[i] = i < p.M ? p.rowc[qrow0 + i] : -INFINITY;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        float* out = p.scores + ((long long)sg.l * p.Hkv + sg.h) * p.T + sg.begin;
+        for (int t = 0; t < sg.nt && ok; ++t) {
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          for (int ch = 0; ch < p.n_chunks; ++ch, ++bit) {
+            const int buf = bit % NBUF;
+            ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = lane_base + buf * BUFCOLS;
+            const int ng = (ch == p.n_chunks - 1 ? p.cw_last : p.cw) / 32;
+            const float* negc = c_sm + ch * p.cw;
+            tmem_ld32(taddr, ra);
+            for (int g = 0; g < ng; g += 2) {
+              tmem_ld_wait(ra);
+              if (g + 1 < ng) tmem_ld32(taddr + (g + 1) * 32, rb);
+              if (p.reduce == SPEC_REDUCE_MAX) prob_accumulate<true>(ra, negc + g * 32, p.a, acc);
+              else                             prob_accumulate<false>(ra, negc + g * 32, p.a, acc);
+              if (g + 1 < ng) {
+                tmem_ld_wait(rb);
+                if (g + 2 < ng) tmem_ld32(taddr + (g + 2) * 32, ra);
+                if (p.reduce == SPEC_REDUCE_MAX) prob_accumulate<true>(rb, negc + (g + 1) * 32, p.a, acc);
+                else                             prob_accumulate<false>(rb, negc + (g + 1) * 32, p.a, acc);
+              }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&t_empty[buf]);
+          }
+          if (!ok) break;
+          const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
+          if (key < sg.n) {
+            out[key] = p.reduce == SPEC_REDUCE_MAX ? fmaxf(fmaxf(acc[0], acc[1]), fmaxf(acc[2], acc[3]))
+                                                   : (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          }
+        }
+      }
+    }
+  }
+
+  if (*abort_flag) {
+    if (tid == 0) report(p.status, SPEC_ERR_TIMEOUT);
+    __nanosleep(200000);                                     // let copies already in flight land
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
+// Combines the per-segment statistics of every query row into its softmax constant.
+__global__ void __launch_bounds__(128) merge_kernel(const ScoreParams p, int n_ctas) {
+  __shared__ int sh_before, sh_total;
+  const int unit = blockIdx.x;
+  const int lh = unit / p.n_seq, s = unit % p.n_seq;
+  if (threadIdx.x == 0) { sh_before = 0; sh_total = 0; }
+  __syncthreads();
+  int before = 0, total = 0;
+  for (int i = threadIdx.x; i < p.n_seq; i += blockDim.x) {
+    int b, n;
+    seq_range(p.cu, p.n_in, i, b, n);
+    const int tiles = (n + kTileKeys - 1) / kTileKeys;
+    total += tiles;
+    if (i < s) before += tiles;
+  }
+  atomicAdd(&sh_before, before);
+  atomicAdd(&sh_total, total);
+  __syncthreads();
+  int b, n;
+  seq_range(p.cu, p.n_in, s, b, n);
+  const int tiles = (n + kTileKeys - 1) / kTileKeys;
+  if (tiles == 0) return;
+  const long long TT = sh_total;
+  const long long N = (long long)p.L * p.Hkv * TT;
+  const long long P = (N + n_ctas - 1) / n_ctas;
+  const long long u0 = (long long)lh * TT + sh_before;
+  const int b0 = (int)(u0 / P), b1 = (int)((u0 + tiles - 1) / P);
+  const int l = lh / p.Hkv, h = lh % p.Hkv;
+  const int qrow0 = ((s * p.L + l) * p.Hq + h * p.G) * p.R;
+  for (int i = threadIdx.x; i < p.M; i += blockDim.x) {
+    float m = -INFINITY;
+    for (int c = b0; c <= b1; ++c) m = fmaxf(m, p.partial[((size_t)(unit + c) * p.M + i) * 2]);
+    float z = 0.f;
+    for (int c = b0; c <= b1; ++c) {
+      const float pm = p.partial[((size_t)(unit + c) * p.M + i) * 2];
+      const float pz = p.partial[((size_t)(unit + c) * p.M + i) * 2 + 1];
+      if (pm > -INFINITY) z += pz * exp2f(pm - m);
+    }
+    float c = m + log2f(z);
+    if (p.row_weight) c -= log2f(p.row_weight[i % p.R]);
+    p.rowc[qrow0 + i] = -c;
+  }
+}
+
+// ------------------------------------------------------------------ host side ---------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+}  // namespace spec
+
+SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void* k, const float* row_weight,
+                               int32_t reduce, int32_t causal_window, float* scores_out, void* workspace,
+                               size_t workspace_bytes, int32_t* status_word, void* stream) {
+  using namespace spec;
+  int rc = check_problem(pr);
+  if (rc != SPEC_OK) return rc;
+  if (!q || !k || !scores_out) return fail(SPEC_ERR_BAD_ARG, "q, k and scores_out must not be NULL");
+  if (reduce != SPEC_REDUCE_SUM && reduce != SPEC_REDUCE_MAX) return fail(SPEC_ERR_BAD_ARG, "reduce=%d is not a spec_reduce value", reduce);
+  if (causal_window != 0) return fail(SPEC_ERR_NOT_IMPLEMENTED, "causal_window=1 is not implemented yet");
+  if (!(pr->softmax_scale > 0.f) || !(pr->softmax_scale < 1e30f)) return fail(SPEC_ERR_BAD_ARG, "softmax_scale must be positive and finite");
+  if (!aligned16(q) || !aligned16(k)) return fail(SPEC_ERR_ALIGNMENT, "q and k must be 16-byte aligned");
+  const int d = pr->head_dim;
+  if (pr->k_stride_token < d || pr->k_stride_head < d || pr->k_stride_layer < d ||
+      (pr->k_stride_token * 2) % 16 || (pr->k_stride_head * 2) % 16 || (pr->k_stride_layer * 2) % 16)
+    return fail(SPEC_ERR_ALIGNMENT, "K strides must be multiples of 8 elements and at least head_dim");
+  const int R = pr->n_lookahead + pr->n_window;
+  const int G = pr->n_q_heads / pr->n_kv_heads;
+  const int M = G * R;
+  const int M_pad = (M + 127) / 128 * 128;
+  if ((int64_t)M_pad * d > 81920 || M_pad / 128 > kMaxMTiles)
+    return fail(SPEC_ERR_UNSUPPORTED, "G*R=%d query rows per KV head at head_dim=%d exceed the resident-query limit (G*R*head_dim <= 81920)", M, d);
+  const WorkspacePlan wp = plan_workspace(pr);
+  if (!workspace || workspace_bytes < wp.total)
+    return fail(SPEC_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", workspace_bytes, wp.total);
+  rc = check_device();
+  if (rc != SPEC_OK) return rc;
+  const int64_t tokens = pr->cu_seqlens ? pr->total_tokens : pr->n_in;
+  if (tokens == 0) return SPEC_OK;
+
+  EncodeTiledFn encode = encode_fn();
+  if (!encode) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+
+  CUtensorMap tm_q, tm_k;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)pr->n_seq * pr->n_layers * pr->n_q_heads * R};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t es[2] = {1, 1};
+    CUresult r = encode(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(SPEC_ERR_CUDA, "tensor map for q could not be encoded (CUresult %d)", (int)r);
+  }
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)pr->total_tokens, (cuuint64_t)pr->n_kv_heads, (cuuint64_t)pr->n_layers};
+    const cuuint64_t strides[3] = {(cuuint64_t)pr->k_stride_token * 2, (cuuint64_t)pr->k_stride_head * 2, (cuuint64_t)pr->k_stride_layer * 2};
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = encode(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(SPEC_ERR_CUDA, "tensor map for k could not be encoded (CUresult %d)", (int)r);
+  }
+
+  ScoreParams p;
+  p.cu = pr->cu_seqlens;
+  p.row_weight = row_weight;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  p.partial = reinterpret_cast<float*>(ws + wp.partial_off);
+  p.rowc = reinterpret_cast<float*>(ws + wp.rowc_off);
+  p.scores = scores_out;
+  p.status = status_word;
+  p.T = pr->total_tokens;
+  p.n_in = pr->n_in; p.n_seq = pr->n_seq; p.L = pr->n_layers; p.Hq = pr->n_q_heads; p.Hkv = pr->n_kv_heads;
+  p.G = G; p.R = R; p.M = M; p.M_pad = M_pad; p.d = d;
+  const int M32 = (M + 31) / 32 * 32;
+  p.n_chunks = (M32 + 255) / 256;
+  p.cw = ((M32 + p.n_chunks - 1) / p.n_chunks + 31) / 32 * 32;
+  p.cw_last = M32 - (p.n_chunks - 1) * p.cw;
+  p.reduce = reduce;
+  p.a = (float)((double)pr->softmax_scale * 1.4426950408889634);
+  p.q_bytes = (uint32_t)M_pad * d * 2;
+  p.stage_bytes = (uint32_t)kTileKeys * d * 2;
+  const int small = M_pad * 4 + (pr->n_seq + 1) * 4 + 8 + kNumBars * 8 + 16;
+  const int smem_max = 227 * 1024;
+  int stages = (smem_max - (int)p.q_bytes - small) / (int)p.stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return fail(SPEC_ERR_UNSUPPORTED, "not enough shared memory for two key stages (M=%d, head_dim=%d)", M, d);
+  p.n_stages = stages;
+  int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
+  if (smem < 120 * 1024) smem = 120 * 1024;               // one CTA per SM: each CTA owns the whole TMEM
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_ctas = wp.score_ctas;
+  const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
+  SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  score_kernel<1><<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);
+  SPEC_CUDA_OK(cudaGetLastError());
+  score_kernel<2><<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  return SPEC_OK;
+}

@@ -1,0 +1,445 @@
+// Pooling + exact top-C selection (Algorithm 1 lines 10 and 13) and the SpecPC keep set
+// (Algorithm 2 lines 7-10).
+//
+// One CTA owns one (sequence, layer, KV head) unit (SpecPC: one sequence).  Pooled values
+// are turned into order-preserving 32-bit keys; the C-th largest key is found by an MSB-first
+// radix select with shared-memory histograms (one private histogram per warp, run-length
+// aggregated updates), and the winners are emitted in ascending position by a chunked block
+// scan, which also resolves ties at the threshold in favour of the lower position.  Keys are
+// kept in shared memory when the unit fits; longer units recompute them from global memory in
+// every pass.
+#include "common.cuh"
+
+namespace spec {
+
+constexpr int kSelThreads = 512;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelVec = 4;                       // consecutive positions per thread in the ordered pass
+constexpr int kSmemLimit = 227 * 1024;
+
+// Monotone map float -> uint32 (larger float <=> larger key), valid for any sign.
+__device__ __forceinline__ uint32_t to_key(float v) {
+  const uint32_t b = __float_as_uint(v);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Pooled value of position j over the eligible range [0, e).
+__device__ __forceinline__ float pooled_at(const float* __restrict__ s, int e, int j, int pool, int k) {
+  int lo = j - (k >> 1);
+  int hi = lo + k - 1;
+  lo = lo < 0 ? 0 : lo;
+  hi = hi > e - 1 ? e - 1 : hi;
+  if (pool == SPEC_POOL_MAX) {
+    float m = s[lo];
+    for (int t = lo + 1; t <= hi; ++t) m = fmaxf(m, s[t]);
+    return m;
+  }
+  float a = 0.f;
+  for (int t = lo; t <= hi; ++t) a += s[t];
+  return a / (float)k;
+}
+
+// Key source: shared-memory resident keys, or recomputation from the scores.
+struct KeySource {
+  const uint32_t* keys;       // non-NULL when resident
+  const float* scores;
+  int e, pool, k;
+  __device__ __forceinline__ uint32_t operator()(int j) const {
+    return keys ? keys[j] : to_key(pooled_at(scores, e, j, pool, k));
+  }
+};
+
+struct SelectScratch {
+  uint32_t* hist;             // [kSelWarps][256]
+  int* misc;                  // [2*kSelWarps + 8]
+};
+
+// Finds the key T of the `need`-th largest element of key(0..e): count(key > T) < need <=
+// count(key >= T).  Returns T and need_eq = need - count(key > T) (how many elements equal to
+// T belong to the selection).  Requires 1 <= need <= e.  All threads of the CTA must call.
+__device__ void radix_select(const KeySource& key, int e, int need, const SelectScratch& sc,
+                             uint32_t& T_out, int& need_eq_out) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t prefix = 0, mask = 0;
+  int remaining = need;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < kSelWarps * 256; i += kSelThreads) sc.hist[i] = 0;
+    __syncthreads();
+    uint32_t* myh = sc.hist + warp * 256;
+    int run_d = -1, run_c = 0;
+    for (int j = tid; j < e; j += kSelThreads) {
+      const uint32_t kk = key(j);
+      if ((kk & mask) == prefix) {
+        const int dg = (kk >> shift) & 255;
+        if (dg == run_d) {
+          ++run_c;
+        } else {
+          if (run_c) atomicAdd(&myh[run_d], (uint32_t)run_c);
+          run_d = dg;
+          run_c = 1;
+        }
+      }
+    }
+    if (run_c) atomicAdd(&myh[run_d], (uint32_t)run_c);
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t tot = 0;
+#pragma unroll
+      for (int w = 0; w < kSelWarps; ++w) tot += sc.hist[w * 256 + tid];
+      sc.hist[tid] = tot;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the digit.
+      uint32_t b[8], s = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { b[i] = sc.hist[lane * 8 + i]; s += b[i]; }
+      uint32_t suf = s;                                  // inclusive suffix sum over lanes >= lane
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += t;
+      }
+      const uint32_t above = suf - s;                    // elements in bins of higher lanes
+      if (above < (uint32_t)remaining && (uint32_t)remaining <= suf) {
+        uint32_t cum = above;
+        int dg = 7;
+        for (; dg > 0; --dg) {
+          if (cum + b[dg] >= (uint32_t)remaining) break;
+          cum += b[dg];
+        }
+        sc.misc[0] = lane * 8 + dg;
+        sc.misc[1] = (int)cum;                           // elements strictly above the digit
+      }
+    }
+    __syncthreads();
+    const int dg = sc.misc[0];
+    remaining -= sc.misc[1];
+    prefix |= (uint32_t)dg << shift;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  T_out = prefix;
+  need_eq_out = remaining;
+}
+
+// Visits, in ascending position, every selected position j of [0, e): key > T, or key == T and
+// fewer than need_eq equal keys precede it.  emit(rank, j) receives the 0-based rank in the
+// ascending output.  Returns the number of selected positions.  All threads must call.
+template <class Emit>
+__device__ int ordered_emit(const KeySource& key, int e, uint32_t T, int need_eq, const SelectScratch& sc, Emit emit) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int base_gt = 0, base_eq = 0;
+  int* wg = sc.misc + 8;
+  int* we = sc.misc + 8 + kSelWarps;
+  for (int c0 = 0; c0 < e; c0 += kSelThreads * kSelVec) {
+    const int j0 = c0 + tid * kSelVec;
+    uint32_t kk[kSelVec];
+    int gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelVec; ++i) {
+      const int j = j0 + i;
+      kk[i] = j < e ? key(j) : 0u;
+      if (j < e) { gt += kk[i] > T; eq += kk[i] == T; }
+    }
+    int sgt = gt, seq = eq;                               // inclusive warp scans
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, sgt, o);
+      const int b = __shfl_up_sync(0xffffffffu, seq, o);
+      if (lane >= o) { sgt += a; seq += b; }
+    }
+    if (lane == 31) { wg[warp] = sgt; we[warp] = seq; }
+    __syncthreads();
+    int pre_gt = base_gt + sgt - gt, pre_eq = base_eq + seq - eq, tot_gt = 0, tot_eq = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+      const int a = wg[w], b = we[w];
+      if (w < warp) { pre_gt += a; pre_eq += b; }
+      tot_gt += a;
+      tot_eq += b;
+    }
+#pragma unroll
+    for (int i = 0; i < kSelVec; ++i) {
+      const int j = j0 + i;
+      if (j < e) {
+        if (kk[i] > T) {
+          emit(pre_gt + min(pre_eq, need_eq), j);
+          ++pre_gt;
+        } else if (kk[i] == T) {
+          if (pre_eq < need_eq) emit(pre_gt + pre_eq, j);
+          ++pre_eq;
+        }
+      }
+    }
+    base_gt += tot_gt;
+    base_eq += tot_eq;
+    __syncthreads();
+  }
+  return base_gt + min(base_eq, need_eq);
+}
+
+struct TopkParams {
+  const float* scores;
+  const int32_t* cu;
+  int32_t* idx_out;
+  int32_t* count_out;
+  int64_t T;
+  int n_in, L, H, pool, pool_k, c_max, n_forced, cap;
+};
+
+__global__ void __launch_bounds__(kSelThreads) pool_topk_kernel(TopkParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  SelectScratch sc;
+  sc.hist = reinterpret_cast<uint32_t*>(smem_raw);
+  sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
+  uint32_t* keys = reinterpret_cast<uint32_t*>(sc.misc + 2 * kSelWarps + 8);
+
+  const int unit = blockIdx.x;
+  const int h = unit % p.H, l = (unit / p.H) % p.L, s = unit / (p.H * p.L);
+  int begin, n;
+  seq_range(p.cu, p.n_in, s, begin, n);
+  const int forced = min(p.n_forced, n);
+  const int e = n - forced;
+  const int take = min(p.c_max - forced, e);
+  int32_t* idx = p.idx_out + (int64_t)unit * p.c_max;
+  const int tid = threadIdx.x;
+
+  if (take > 0 && take < e) {
+    KeySource key;
+    key.scores = p.scores + ((int64_t)l * p.H + h) * p.T + begin;
+    key.e = e; key.pool = p.pool; key.k = p.pool_k;
+    key.keys = nullptr;
+    if (e <= p.cap) {
+      for (int j = tid; j < e; j += kSelThreads) keys[j] = key(j);
+      key.keys = keys;
+      __syncthreads();
+    }
+    uint32_t T;
+    int need_eq;
+    radix_select(key, e, take, sc, T, need_eq);
+    ordered_emit(key, e, T, need_eq, sc, [&](int rank, int j) { idx[rank] = j; });
+  } else {
+    for (int c = tid; c < take; c += kSelThreads) idx[c] = c;      // every eligible position is kept
+  }
+  for (int c = take + tid; c < p.c_max; c += kSelThreads) idx[c] = (c - take < forced) ? e + (c - take) : -1;
+  if (p.count_out && tid == 0) p.count_out[unit] = take + forced;
+}
+
+// ---------------------------------------------------------------------- SpecPC ------
+
+// Token score: reduction over all layers and KV heads, in (layer, head) order.
+__global__ void __launch_bounds__(256) token_reduce_kernel(const float* __restrict__ scores, float* __restrict__ tok,
+                                                           int64_t T, int n_vec, int reduce) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const float* src = scores + t;
+  float acc = reduce == SPEC_REDUCE_SUM ? 0.f : -INFINITY;
+  int i = 0;
+  for (; i + 8 <= n_vec; i += 8) {
+    float x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = __ldg(src + (int64_t)(i + u) * T);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc = reduce == SPEC_REDUCE_SUM ? acc + x[u] : fmaxf(acc, x[u]);
+  }
+  for (; i < n_vec; ++i) {
+    const float x = __ldg(src + (int64_t)i * T);
+    acc = reduce == SPEC_REDUCE_SUM ? acc + x : fmaxf(acc, x);
+  }
+  tok[t] = acc;
+}
+
+struct KeepParams {
+  const float* tok;
+  const int32_t* cu;
+  int32_t* keep_out;
+  int32_t* n_keep_out;
+  int n_in, pool, pool_k, c_max, n_neighbor, n_forced, keep_capacity, cap, bitmap_words;
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(kSelThreads) specpc_keep_kernel(KeepParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  SelectScratch sc;
+  sc.hist = reinterpret_cast<uint32_t*>(smem_raw);
+  sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(sc.misc + 2 * kSelWarps + 8);
+  uint32_t* keys = bitmap + p.bitmap_words;
+
+  const int s = blockIdx.x;
+  int begin, n;
+  seq_range(p.cu, p.n_in, s, begin, n);
+  const int forced = min(p.n_forced, n);
+  const int e = n - forced;
+  const int take = min(p.c_max, e);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int32_t* keep = p.keep_out + (int64_t)s * p.keep_capacity;
+  const int n_words = (n + 31) >> 5;
+
+  for (int w = tid; w < n_words; w += kSelThreads) bitmap[w] = 0;
+  __syncthreads();
+
+  auto mark = [&](int lo, int hi) {                       // set bits lo..hi (inclusive)
+    for (int w = lo >> 5; w <= (hi >> 5); ++w) {
+      const int b0 = max(lo, w << 5) & 31, b1 = min(hi, (w << 5) + 31) & 31;
+      const uint32_t m = (0xffffffffu >> (31 - b1)) & (0xffffffffu << b0);
+      atomicOr(&bitmap[w], m);
+    }
+  };
+
+  if (take > 0 && take < e) {
+    KeySource key;
+    key.scores = p.tok + begin;
+    key.e = e; key.pool = p.pool; key.k = p.pool_k;
+    key.keys = nullptr;
+    if (e <= p.cap) {
+      for (int j = tid; j < e; j += kSelThreads) keys[j] = key(j);
+      key.keys = keys;
+      __syncthreads();
+    }
+    uint32_t T;
+    int need_eq;
+    radix_select(key, e, take, sc, T, need_eq);
+    const int nb = p.n_neighbor;
+    ordered_emit(key, e, T, need_eq, sc, [&](int, int j) { mark(max(j - nb, 0), min(j + nb, e - 1)); });
+  } else if (take > 0) {
+    for (int w = tid; w < ((e + 31) >> 5); w += kSelThreads) {
+      const int hi = min(e - 1, (w << 5) + 31);
+      mark(w << 5, hi);
+    }
+  }
+  __syncthreads();
+  if (forced > 0) {
+    for (int j = e + tid; j < n; j += kSelThreads) mark(j, j);
+    __syncthreads();
+  }
+
+  // Ordered extraction of the set bits: every thread owns a run of consecutive words.
+  const int wpt = (n_words + kSelThreads - 1) / kSelThreads;
+  const int w0 = tid * wpt, w1 = min(w0 + wpt, n_words);
+  int cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+  int sc_incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int a = __shfl_up_sync(0xffffffffu, sc_incl, o);
+    if (lane >= o) sc_incl += a;
+  }
+  int* wt = sc.misc + 8;
+  if (lane == 31) wt[warp] = sc_incl;
+  __syncthreads();
+  int pos = sc_incl - cnt, total = 0;
+#pragma unroll
+  for (int w = 0; w < kSelWarps; ++w) {
+    if (w < warp) pos += wt[w];
+    total += wt[w];
+  }
+  for (int w = w0; w < w1; ++w) {
+    uint32_t bits = bitmap[w];
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (pos < p.keep_capacity) keep[pos] = (w << 5) + b;
+      ++pos;
+    }
+  }
+  if (total > p.keep_capacity && tid == 0) report(p.status, SPEC_ERR_BAD_ARG);
+  const int kept = min(total, p.keep_capacity);
+  for (int c = kept + tid; c < p.keep_capacity; c += kSelThreads) keep[c] = -1;
+  if (tid == 0) p.n_keep_out[s] = kept;
+}
+
+static int select_smem_bytes(int max_len, int bitmap_words, int* cap_out) {
+  const int fixed = kSelWarps * 256 * 4 + (2 * kSelWarps + 8) * 4 + bitmap_words * 4;
+  int cap = (kSmemLimit - fixed) / 4;
+  cap &= ~3;
+  if (cap < 0) cap = 0;
+  int want = max_len <= cap ? max_len : 0;                 // longer units stream from global memory
+  *cap_out = want;
+  return fixed + want * 4;
+}
+
+static int check_pool_args(int pool, int pool_k, int c_max, int n_forced_tail) {
+  if (pool != SPEC_POOL_MAX && pool != SPEC_POOL_AVG) return fail(SPEC_ERR_BAD_ARG, "pool=%d is not a spec_pool value", pool);
+  if (pool_k < 1 || pool_k > 255) return fail(SPEC_ERR_BAD_ARG, "pool_k=%d outside [1, 255]", pool_k);
+  if (c_max < 1) return fail(SPEC_ERR_BAD_ARG, "c_max=%d must be >= 1", c_max);
+  if (n_forced_tail < 0) return fail(SPEC_ERR_BAD_ARG, "n_forced_tail=%d is negative", n_forced_tail);
+  return SPEC_OK;
+}
+
+}  // namespace spec
+
+SPEC_EXPORT int32_t spec_pool_topk(const spec_problem* pr, const float* scores, int32_t pool, int32_t pool_k,
+                                   int32_t c_max, int32_t n_forced_tail, int32_t* idx_out, int32_t* count_out,
+                                   void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
+  using namespace spec;
+  (void)workspace; (void)workspace_bytes; (void)status_word;
+  int rc = check_problem(pr);
+  if (rc != SPEC_OK) return rc;
+  if (!scores || !idx_out) return fail(SPEC_ERR_BAD_ARG, "scores and idx_out must not be NULL");
+  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);
+  if (rc != SPEC_OK) return rc;
+  if (n_forced_tail > c_max) return fail(SPEC_ERR_BAD_ARG, "n_forced_tail=%d exceeds c_max=%d", n_forced_tail, c_max);
+  rc = check_device();
+  if (rc != SPEC_OK) return rc;
+
+  TopkParams p;
+  p.scores = scores; p.cu = pr->cu_seqlens; p.idx_out = idx_out; p.count_out = count_out;
+  p.T = pr->total_tokens; p.n_in = pr->n_in; p.L = pr->n_layers; p.H = pr->n_kv_heads;
+  p.pool = pool; p.pool_k = pool_k; p.c_max = c_max; p.n_forced = n_forced_tail;
+  const int smem = select_smem_bytes(max_seq_len(pr), 0, &p.cap);
+  SPEC_CUDA_OK(cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
+  pool_topk_kernel<<<n_units, kSelThreads, smem, static_cast<cudaStream_t>(stream)>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  return SPEC_OK;
+}
+
+SPEC_EXPORT int32_t specpc_token_select(const spec_problem* pr, const float* scores, int32_t layer_head_reduce,
+                                        int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,
+                                        int32_t n_forced_tail, int32_t* keep_out, int32_t keep_capacity,
+                                        int32_t* n_keep_out, void* workspace, size_t workspace_bytes,
+                                        int32_t* status_word, void* stream) {
+  using namespace spec;
+  int rc = check_problem(pr);
+  if (rc != SPEC_OK) return rc;
+  if (!scores || !keep_out || !n_keep_out) return fail(SPEC_ERR_BAD_ARG, "scores, keep_out and n_keep_out must not be NULL");
+  if (layer_head_reduce != SPEC_REDUCE_SUM && layer_head_reduce != SPEC_REDUCE_MAX)
+    return fail(SPEC_ERR_BAD_ARG, "layer_head_reduce=%d is not a spec_reduce value", layer_head_reduce);
+  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);
+  if (rc != SPEC_OK) return rc;
+  if (n_neighbor < 0) return fail(SPEC_ERR_BAD_ARG, "n_neighbor=%d is negative", n_neighbor);
+  const int max_len = max_seq_len(pr);
+  const int64_t worst = (int64_t)c_max * (2 * (int64_t)n_neighbor + 1) + n_forced_tail;
+  const int64_t need_cap = worst < max_len ? worst : max_len;
+  if (keep_capacity < need_cap)
+    return fail(SPEC_ERR_BAD_ARG, "keep_capacity=%d is below the worst case %lld", keep_capacity, (long long)need_cap);
+  const WorkspacePlan wp = plan_workspace(pr);
+  if (!workspace || workspace_bytes < wp.total)
+    return fail(SPEC_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", workspace_bytes, wp.total);
+  const int bitmap_words = (max_len + 31) / 32 + 1;
+  if ((int64_t)bitmap_words * 4 > 160 * 1024)
+    return fail(SPEC_ERR_UNSUPPORTED, "sequences longer than %d tokens are not supported by specpc_token_select", 160 * 1024 * 8);
+  rc = check_device();
+  if (rc != SPEC_OK) return rc;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* tok = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + wp.token_off);
+  const int64_t T = pr->total_tokens;
+  if (T > 0) {
+    token_reduce_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(scores, tok, T, pr->n_layers * pr->n_kv_heads,
+                                                                     layer_head_reduce);
+    SPEC_CUDA_OK(cudaGetLastError());
+  }
+  KeepParams p;
+  p.tok = tok; p.cu = pr->cu_seqlens; p.keep_out = keep_out; p.n_keep_out = n_keep_out;
+  p.n_in = pr->n_in; p.pool = pool; p.pool_k = pool_k; p.c_max = c_max; p.n_neighbor = n_neighbor;
+  p.n_forced = n_forced_tail; p.keep_capacity = keep_capacity; p.bitmap_words = bitmap_words;
+  p.status = status_word;
+  const int smem = select_smem_bytes(max_len, bitmap_words, &p.cap);
+  SPEC_CUDA_OK(cudaFuncSetAttribute(specpc_keep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  specpc_keep_kernel<<<(unsigned)pr->n_seq, kSelThreads, smem, st>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  return SPEC_OK;
+}
