@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the lookahead-importance hot path: one step = spec_score -> spec_pool_topk ->
+spec_compact_kv (SpecPC workload: spec_score -> specpc_token_select) over ALL layers of one
+synthetic workload.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+metric  : prompt tokens scored + compacted per second (all layers), whole job over N GPUs.
+value   : device-timed (CUDA events), inputs resident in HBM.
+e2e     : same metric with the host->device copy of Q/K/V from pinned memory and the
+          device->host read of the selection inside the timed region.
+roofline: the scoring call (two tensor-core passes) against the measured bf16 peak.
+cpu_baseline: the fp64 oracle timed on the host cores on a bounded sample (rank 0, N = 1).
+With N > 1 every rank runs the same per-GPU workload (weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "prompt_tokens_scored_and_compacted_per_s_all_layers"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "of measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "of fallback"
+
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="workload index (1 = the configuration the metric is quoted on)")
+    ap.add_argument("--layers", type=int, default=0, help="debug/profiling only: run the first LAYERS layers")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    return ap.parse_args(argv)
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's time (the job finishes when the last rank does)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(tokens_per_rank: int, steps: int, world: int, max_ms_total: float) -> float:
+    """Whole-job throughput: every rank processed `tokens_per_rank` prompt tokens per step."""
+    return world * tokens_per_rank * steps / (max_ms_total * 1e-3)
+
+
+# ------------------------------------------------------------------ clocks ------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is not None:
+            time.sleep(0.06)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        try:
+            self.file.flush()
+            self.file.seek(0)
+            rows = [r.strip().split(",") for r in self.file.read().strip().splitlines() if r.strip()]
+            sm = [float(r[0]) for r in rows if len(r) >= 8]
+            if sm:
+                hi = max(sm)
+                load = [x for x in sm if x >= 0.5 * hi] or sm
+                out["sm_mhz"] = statistics.median(load)
+                out["sm_max_mhz"] = float(rows[0][1])
+                out["samples"] = len(sm)
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                for i, n in enumerate(names):
+                    if any(r[4 + i].strip().lower().startswith("active") for r in rows if len(r) >= 8):
+                        out["reasons"].append(n)
+        except Exception:
+            pass
+        finally:
+            try:
+                self.file.close()
+                os.unlink(self.file.name)
+            except Exception:
+                pass
+        return out
+
+
+# ------------------------------------------------------------------ workload ----------
+
+class State:
+    """Device-resident inputs, outputs and scratch of one workload."""
+
+    def __init__(self, B, W, w, device, layers):
+        import torch
+        self.B, self.w, self.device = B, w, device
+        self.L = len(layers)
+        self.q, self.k, self.v = W.gen_layers(w, layers, device, want_v=(w.n_neighbor == 0))
+        self.cu = W.cu_seqlens(w)
+        self.T = self.cu[-1]
+        self.cu_t = torch.tensor(self.cu, dtype=torch.int32, device=device) if w.n_seq > 1 else None
+        self.pr = B.make_problem(n_layers=self.L, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                                 head_dim=w.head_dim, n_lookahead=w.n_lookahead, n_window=w.n_window,
+                                 softmax_scale=w.scale, total_tokens=self.T,
+                                 n_in=(w.n_in if w.n_in is not None else max(W.seq_lens(w))), n_seq=w.n_seq,
+                                 cu_seqlens=self.cu_t, k=self.k, v=self.v)
+        self.ws = torch.empty(B.spec_workspace_bytes(self.pr), dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.scores = torch.empty((self.L, w.n_kv_heads, self.T), dtype=torch.float32, device=device)
+        self.specpc = w.n_neighbor > 0
+        if self.specpc:
+            self.cap = min(max(W.seq_lens(w)), w.c_max * (2 * w.n_neighbor + 1))
+            self.keep = torch.empty((w.n_seq, self.cap), dtype=torch.int32, device=device)
+            self.n_keep = torch.empty((w.n_seq,), dtype=torch.int32, device=device)
+            self.results = [self.keep, self.n_keep]
+        else:
+            self.idx = torch.empty((w.n_seq, self.L, w.n_kv_heads, w.c_max), dtype=torch.int32, device=device)
+            self.cnt = torch.empty((w.n_seq, self.L, w.n_kv_heads), dtype=torch.int32, device=device)
+            self.bt = None
+            if w.page_size:
+                self.bt = W.block_table(w, device)
+                self.n_pages = self.bt.numel()
+                shape = (self.L, self.n_pages, w.n_kv_heads, w.page_size, w.head_dim)
+            else:
+                shape = (w.n_seq, self.L, w.n_kv_heads, w.c_max, w.head_dim)
+            self.k_out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+            self.v_out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+            self.results = [self.idx, self.cnt]
+        self.launches_per_step = 3 + (2 if self.specpc else 2)
+
+    def step(self, events=None):
+        B, w = self.B, self.w
+        if events is not None:
+            events[0].record()
+        B.spec_score(self.pr, self.q, self.k, self.scores, self.ws, status_word=self.status)
+        if events is not None:
+            events[1].record()
+        if self.specpc:
+            B.specpc_token_select(self.pr, self.scores, B.REDUCE_SUM, B.POOL_MAX, w.pool_k, w.c_max, w.n_neighbor, 0,
+                                  self.keep, self.cap, self.n_keep, self.ws, status_word=self.status)
+            if events is not None:
+                events[2].record()
+                events[3].record()
+        else:
+            B.spec_pool_topk(self.pr, self.scores, B.POOL_MAX, w.pool_k, w.c_max, 0, self.idx, self.cnt,
+                             status_word=self.status)
+            if events is not None:
+                events[2].record()
+            if self.bt is not None:
+                B.spec_compact_kv(self.pr, self.k, self.v, self.idx, w.c_max, self.k_out, self.v_out,
+                                  block_table=self.bt, page_size=w.page_size, n_pages=self.n_pages,
+                                  status_word=self.status)
+            else:
+                B.spec_compact_kv(self.pr, self.k, self.v, self.idx, w.c_max, self.k_out, self.v_out,
+                                  status_word=self.status)
+            if events is not None:
+                events[3].record()
+
+
+def algorithmic_work(w, L, tokens):
+    """Algorithmic flops and bytes of one step (the per-unit figures times the units of a launch)."""
+    R, d, C = w.rows, w.head_dim, w.c_max
+    flops_one_pass = 2.0 * L * w.n_q_heads * R * tokens * d
+    k_bytes_one_pass = 2.0 * d * w.n_kv_heads * L * tokens
+    score_bytes = 4.0 * w.n_kv_heads * L * tokens
+    select_bytes = score_bytes + 4.0 * w.n_kv_heads * L * C * w.n_seq
+    gather_bytes = 0.0 if w.n_neighbor else 8.0 * w.n_kv_heads * L * C * d * w.n_seq
+    return {"flops_two_pass": 2 * flops_one_pass, "flops_one_pass": flops_one_pass,
+            "score_hbm_bytes": 2 * k_bytes_one_pass + score_bytes, "select_bytes": select_bytes,
+            "gather_bytes": gather_bytes}
+
+
+def cpu_baseline(W, w, n_layers_sample=1):
+    """The oracle, as it stands, on a bounded sample: the first layer(s) of the workload, all
+    sequences and KV heads, scoring + pooling/top-C + gather (SpecPC: + keep set)."""
+    import numpy as np
+    import torch
+    import oracle
+    oracle.build()
+    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    layers = list(range(min(n_layers_sample, w.n_layers)))
+    q, k, v = W.gen_layers(w, layers, "cpu", want_v=(w.n_neighbor == 0))
+    cu = W.cu_seqlens(w)
+    qb, kb = bits(q), bits(k)
+    vb = bits(v) if v is not None else None
+    t0 = time.perf_counter()
+    sc = oracle.spec_score(qb, kb, cu, w.n_lookahead, w.n_window, w.scale)
+    if w.n_neighbor:
+        oracle.specpc_select(sc, cu, oracle.SUM, oracle.POOL_MAX, w.pool_k, w.c_max, w.n_neighbor, 0)
+    else:
+        idx, _, _, _ = oracle.pool_topk(sc, cu, oracle.POOL_MAX, w.pool_k, w.c_max)
+        oracle.compact(kb, cu, idx)
+        oracle.compact(vb, cu, idx)
+    dt = time.perf_counter() - t0
+    tokens = cu[-1]
+    value = tokens / (dt * w.n_layers / len(layers))
+    return {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%d of %d layers, all sequences and KV heads, %.1f s wall; scaled by layers" %
+                      (len(layers), w.n_layers, dt)}, dt
+
+
+def run_reference(args, W, w):
+    """Reference arm: the CPU oracle timed per step on a bounded sample (one layer)."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    times = []
+    last = None
+    for i in range(args.warmup + args.steps):
+        last, dt = cpu_baseline(W, w, 1)
+        if i >= args.warmup:
+            times.append(dt)
+        if sum(times) > 150:                      # stay within a few minutes on slow hosts
+            break
+    steps = len(times)
+    ms = 1e3 * sum(times) / steps
+    tokens = W.cu_seqlens(w)[-1]
+    value = tokens / (ms * 1e-3 * w.n_layers)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sample": "each step scores, selects and gathers 1 of %d layers on the host; "
+                       "value is scaled to all layers" % w.n_layers},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    from paper_2506_08373_b200 import workloads as W
+    w = W.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, W, w)
+        return 0
+
+    import torch
+    from paper_2506_08373_b200 import binding as B
+    B.lib()                                            # fails loudly when the CUDA library is missing
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    layers = list(range(args.layers if args.layers else w.n_layers))
+    st = State(B, W, w, device, layers)
+    tokens = st.T
+    K, Wm = args.steps, max(args.warmup, 3) if not args.layers else args.warmup
+
+    for _ in range(Wm):
+        st.step()
+    torch.cuda.synchronize()
+    assert st.status.item() == 0, "device-side error status %d" % st.status.item()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    end = torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    for i in range(K):
+        st.step(ev[i])
+    end.record()
+    torch.cuda.synchronize()
+    total_ms = ev[0][0].elapsed_time(end)
+    if world > 1:
+        torch.distributed.barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = max_over_ranks(total_ms, device)
+    assert st.status.item() == 0
+    t_score = sum(e[0].elapsed_time(e[1]) for e in ev) / K
+    t_select = sum(e[1].elapsed_time(e[2]) for e in ev) / K
+    t_gather = sum(e[2].elapsed_time(e[3]) for e in ev) / K
+
+    peaks, peak_src = load_peaks()
+    work = algorithmic_work(w, st.L, tokens)
+    tf = work["flops_two_pass"] / (t_score * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "spec_score: score_kernel<1> + merge + score_kernel<2>",
+                "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                "peak_source": peak_src + " (burst cuBLAS bf16)", "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+                "achieved_one_contraction": tf / 2, "ms": t_score, "traffic": None}
+    hbm_bytes = work["select_bytes"] + work["gather_bytes"]
+    gbs = hbm_bytes / ((t_select + t_gather) * 1e-3) / 1e9
+    roofline_hbm = {"bound": "hbm", "kernel": "pool_topk_kernel + compact_kernel" if not st.specpc else "token_reduce + specpc_keep",
+                    "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                    "peak_source": peak_src + " (copy)", "ms_select": t_select, "ms_gather": t_gather,
+                    "gather_gbs": (work["gather_bytes"] / (t_gather * 1e-3) / 1e9) if t_gather > 0 and work["gather_bytes"] else None,
+                    "traffic": None}
+
+    line = {"metric": METRIC, "value": job_value(tokens, K, world, total_ms), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": Wm, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name + ("" if not args.layers else " (first %d layers only: NOT the quoted configuration)" % args.layers),
+                       "n_layers": st.L, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                       "tokens_per_step": tokens, "n_seq": w.n_seq, "n_lookahead": w.n_lookahead, "n_window": w.n_window,
+                       "pool_k": w.pool_k, "c_max": w.c_max,
+                       "l2": "inputs larger than L2 (K+V %.2f GB per step)" % ((2 if st.v is not None else 1) * st.k.numel() * 2 / 1e9),
+                       "parallelism": "replicated per GPU, no collective" if world > 1 else "single GPU"},
+            "roofline": roofline, "roofline_hbm": roofline_hbm, "gpu_launches": st.launches_per_step * K,
+            "clocks": clocks}
+
+    if rank == 0 and world == 1 and not args.no_e2e:
+        line["e2e"] = run_e2e(st, tokens, min(K, 5))
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["cpu_baseline"], _ = cpu_baseline(W, w, 1)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+def run_e2e(st, tokens, steps):
+    """Host buffers in, selection out: every step copies Q/K/V from pinned host memory, runs the
+    calls and reads the selection back to the host."""
+    import torch
+    dev_in = [t for t in (st.q, st.k, st.v) if t is not None]
+    host_in = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in dev_in]
+    for h, d in zip(host_in, dev_in):
+        h.copy_(d)
+    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in st.results]
+    torch.cuda.synchronize()
+
+    def one():
+        for h, d in zip(host_in, dev_in):
+            d.copy_(h, non_blocking=True)
+        st.step()
+        for h, d in zip(host_out, st.results):
+            h.copy_(d, non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in dev_in),
+            "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in st.results)}
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,372 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Scores within 2e-3 relative + 1e-6 absolute; index sets identical outside the
+tolerance band around the weakest selected score; index work on given scores and the gather
+bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from util import Gpu, assert_index_sets_match, assert_scores_close, bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2506_08373_b200 import binding
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def W():
+    from paper_2506_08373_b200 import workloads
+    return workloads
+
+
+def small(W, **kw):
+    base = W.CONFIGS[1].replace(n_layers=2, n_in=1000, c_max=64, seed=11)
+    return base.replace(**kw)
+
+
+SCORE_CASES = {
+    "c0_tiny": lambda W: (W.CONFIGS[0], [0]),
+    "d128_M384_ragged_tail": lambda W: (small(W), [0, 1]),
+    "d128_M640": lambda W: (small(W, n_lookahead=128, n_in=2500, seed=12), [0]),
+    "d64_M512": lambda W: (W.CONFIGS[3].replace(n_in=3000, n_layers=2, c_max=300, n_planted=8), [0, 1]),
+    "d64_M5_one_head": lambda W: (small(W, head_dim=64, n_q_heads=2, n_kv_heads=2, n_lookahead=3, n_window=2,
+                                        zipf_bias=False, n_in=777), [0]),
+    "d128_M21": lambda W: (small(W, n_q_heads=6, n_kv_heads=2, n_lookahead=4, n_window=3, n_in=300), [0, 1]),
+    "snapkv_no_lookahead": lambda W: (small(W, n_lookahead=0, n_in=513), [0]),
+    "single_key": lambda W: (small(W, n_in=1, zipf_bias=False, planted="singletons", n_planted=0), [0]),
+    "ragged_batch": lambda W: (W.CONFIGS[4].replace(n_layers=2, n_seq=7, len_lo=1, len_hi=900, c_max=64), [0, 1]),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SCORE_CASES))
+def test_score_parity(B, W, oracle, case):
+    w, layers = SCORE_CASES[case](W)
+    g = Gpu(B, W, w, layers)
+    got = g.score().cpu().numpy()
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale)
+    assert_scores_close(got, ref, g.cu)
+    # each softmax row sums to one: the aggregate of a KV head sums to the number of stacked rows
+    for s in range(w.n_seq):
+        if g.cu[s + 1] > g.cu[s]:
+            np.testing.assert_allclose(got[:, :, g.cu[s]:g.cu[s + 1]].astype(np.float64).sum(-1),
+                                       w.group * w.rows, rtol=1e-4)
+
+
+def test_score_ragged_with_empty_and_tile_edge_lengths(B, W, oracle):
+    w = W.CONFIGS[4].replace(n_layers=1, n_seq=8, c_max=32)
+    lens = [1, 127, 128, 129, 0, 700, 256, 5]
+    g = Gpu.__new__(Gpu)
+    g.B, g.w, g.L = B, w, 1
+    T = sum(lens)
+    gen = torch.Generator().manual_seed(5)
+    g.q = torch.randn(8, 1, w.n_q_heads, w.rows, w.head_dim, generator=gen).to(torch.bfloat16).cuda()
+    g.k = torch.randn(1, w.n_kv_heads, T, w.head_dim, generator=gen).to(torch.bfloat16).cuda()
+    g.v = None
+    g.cu = [0] + list(np.cumsum(lens))
+    g.T = T
+    g.cu_t = torch.tensor(g.cu, dtype=torch.int32, device="cuda")
+    g.pr = B.make_problem(n_layers=1, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                          n_lookahead=w.n_lookahead, n_window=w.n_window, softmax_scale=w.scale, total_tokens=T,
+                          n_in=max(lens), n_seq=8, cu_seqlens=g.cu_t, k=g.k)
+    g.ws = torch.empty(B.spec_workspace_bytes(g.pr), dtype=torch.uint8, device="cuda")
+    g.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = g.score().cpu().numpy()
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale)
+    assert_scores_close(got, ref, g.cu)
+    idx, cnt = g.topk(torch.from_numpy(got).cuda(), B.POOL_MAX, 7, 32)
+    oidx, ocnt, _, _ = oracle.pool_topk(got.astype(np.float64), g.cu, oracle.POOL_MAX, 7, 32)
+    np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), ocnt)
+    assert list(ocnt[:, 0, 0]) == [1, 32, 32, 32, 0, 32, 32, 5]
+
+
+def test_score_max_reduce_and_row_weights(B, W, oracle):
+    w = small(W, n_in=600)
+    g = Gpu(B, W, w, [0])
+    rw = torch.linspace(1.0 / w.rows, 1.0, w.rows)
+    rw[3] = 0.0
+    for reduce in (B.REDUCE_SUM, B.REDUCE_MAX):
+        got = g.score(reduce=reduce, row_weight=rw.cuda()).cpu().numpy()
+        ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale,
+                                row_weight=rw.double().numpy(), mode=reduce)
+        assert_scores_close(got, ref, g.cu)
+    got = g.score(reduce=B.REDUCE_MAX).cpu().numpy()
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale, mode=oracle.MAX)
+    assert_scores_close(got, ref, g.cu)
+    assert got.max() <= 1.0 + 1e-5
+
+
+def test_score_token_major_key_layout_and_reproducibility(B, W, oracle):
+    w = small(W, n_in=900)
+    g = Gpu(B, W, w, [0, 1])
+    base = g.score()
+    again = g.score()
+    assert torch.equal(base, again), "scores must be bit-reproducible run to run"
+    kt = g.k.permute(0, 2, 1, 3).contiguous()               # memory order [L, T, Hkv, d]
+    view = kt.permute(0, 2, 1, 3)                           # logical [L, Hkv, T, d] with token-major strides
+    g.pr = B.make_problem(n_layers=2, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                          n_lookahead=w.n_lookahead, n_window=w.n_window, softmax_scale=w.scale,
+                          total_tokens=g.T, n_in=w.n_in, k=view)
+    g.k = view
+    assert torch.equal(g.score(), base)
+
+
+def test_score_rejects_unsupported_shapes(B, W):
+    w = small(W, n_q_heads=64, n_kv_heads=2)               # 32*96 rows per KV head
+    g = Gpu(B, W, w, [0])
+    with pytest.raises(B.SpecError) as e:
+        g.score()
+    assert e.value.code == B.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ selection ---------
+
+def run_topk_case(B, W, oracle, scores, cu, pool, k, c_max, forced, exact=True):
+    L, H, T = scores.shape
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda") if len(cu) > 2 else None   # must outlive the call
+    pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=128, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=T, n_in=int(max(np.diff(cu))), n_seq=len(cu) - 1,
+                        cu_seqlens=cu_t)
+    idx = torch.full((len(cu) - 1, L, H, c_max), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((len(cu) - 1, L, H), -7, dtype=torch.int32, device="cuda")
+    B.spec_pool_topk(pr, torch.from_numpy(scores).cuda(), pool, k, c_max, forced, idx, cnt)
+    torch.cuda.synchronize()
+    oidx, ocnt, pooled, th = oracle.pool_topk(scores.astype(np.float64), cu, pool, k, c_max, forced)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), ocnt)
+    if exact:
+        np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
+    else:
+        gi = idx.cpu().numpy()
+        for s in range(len(cu) - 1):
+            for l in range(L):
+                for h in range(H):
+                    nf = min(forced, cu[s + 1] - cu[s])
+                    e = cu[s + 1] - cu[s] - nf
+                    ge, oe = gi[s, l, h], oidx[s, l, h]
+                    assert_index_sets_match(ge[(ge >= 0) & (ge < e)], oe[(oe >= 0) & (oe < e)],
+                                            pooled[l, h, cu[s]:cu[s + 1]], th[s, l, h])
+
+
+def test_topk_exact_with_ties_runs_and_forced_tail(B, W, oracle):
+    rng = np.random.default_rng(1)
+    # heavy ties: few distinct values, max-pool makes runs of equal keys
+    scores = (rng.integers(0, 5, size=(2, 3, 5000)) / 8).astype(np.float32)
+    run_topk_case(B, W, oracle, scores, [0, 5000], 0, 7, 256, 0)
+    run_topk_case(B, W, oracle, scores, [0, 5000], 0, 7, 256, 32)
+    run_topk_case(B, W, oracle, scores, [0, 1200, 1200, 1210, 5000], 0, 7, 100, 16)
+    run_topk_case(B, W, oracle, np.zeros((1, 1, 3000), np.float32), [0, 3000], 0, 7, 500, 0)   # all equal
+    scores = rng.random((2, 2, 4097)).astype(np.float32) ** 8
+    for k in (1, 3, 7, 13):
+        run_topk_case(B, W, oracle, scores, [0, 4097], 0, k, 1024, 0)
+    run_topk_case(B, W, oracle, scores, [0, 4097], 0, 7, 4096, 0)       # one position dropped
+    run_topk_case(B, W, oracle, scores, [0, 4097], 0, 7, 4097, 0)       # keep all
+    run_topk_case(B, W, oracle, scores, [0, 4097], 0, 7, 5000, 7)       # c_max > n : -1 padding
+    run_topk_case(B, W, oracle, scores, [0, 4097], 0, 7, 1, 0)
+    run_topk_case(B, W, oracle, scores, [0, 4097], 0, 7, 64, 64)        # nothing but the forced tail
+
+
+def test_topk_streaming_regime_long_sequence(B, W, oracle):
+    rng = np.random.default_rng(2)
+    scores = rng.random((1, 2, 70001)).astype(np.float32) ** 6
+    scores[0, 0, ::1000] = 0.75                                          # ties at the top
+    run_topk_case(B, W, oracle, scores, [0, 70001], 0, 7, 2048, 0)
+    run_topk_case(B, W, oracle, scores, [0, 70001], 0, 7, 2048, 32)
+
+
+def test_topk_avg_pool_within_band(B, W, oracle):
+    rng = np.random.default_rng(3)
+    scores = rng.random((1, 2, 3000)).astype(np.float32) ** 4
+    run_topk_case(B, W, oracle, scores, [0, 3000], 1, 7, 128, 0, exact=False)
+    run_topk_case(B, W, oracle, scores, [0, 3000], 1, 13, 128, 8, exact=False)
+
+
+# ------------------------------------------------------------------ compaction --------
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_compact_bit_exact_contiguous_and_paged(B, W, oracle, d):
+    rng = np.random.default_rng(4)
+    L, H, C = 2, 3, 70
+    cu = [0, 300, 300, 1000]
+    T = 1000
+    k = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
+    v = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
+    idx = np.full((3, L, H, C), -1, dtype=np.int32)
+    for s, n in enumerate((300, 0, 700)):
+        for l in range(L):
+            for h in range(H):
+                m = min(n, C - 3)
+                idx[s, l, h, :m] = np.sort(rng.choice(n, m, replace=False)) if n else []
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda")
+    pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=d, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=T, n_in=700, n_seq=3, cu_seqlens=cu_t, k=k, v=v)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    idx_t = torch.from_numpy(idx).cuda()
+    ko = torch.full((3, L, H, C, d), 1.0, dtype=torch.bfloat16, device="cuda")
+    vo = torch.full_like(ko, 1.0)
+    B.spec_compact_kv(pr, k, v, idx_t, C, ko, vo, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    np.testing.assert_array_equal(bits(ko), oracle.compact(bits(k), cu, idx))
+    np.testing.assert_array_equal(bits(vo), oracle.compact(bits(v), cu, idx))
+    # K only
+    ko.fill_(1.0)
+    B.spec_compact_kv(pr, k, None, idx_t, C, ko, None, status_word=status)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(bits(ko), oracle.compact(bits(k), cu, idx))
+    # paged, pages deliberately scattered
+    ps, pps = 16, (C + 15) // 16
+    n_pages = 3 * pps + 2
+    bt = rng.permutation(n_pages)[: 3 * pps].astype(np.int32).reshape(3, pps)
+    kp = torch.from_numpy(np.full((L, n_pages, H, ps, d), 0x7FFF, np.int16)).view(torch.bfloat16).cuda()
+    vp = kp.clone()
+    B.spec_compact_kv(pr, k, v, idx_t, C, kp, vp, block_table=torch.from_numpy(bt).cuda(), page_size=ps,
+                      n_pages=n_pages, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for src, pool in ((k, kp), (v, vp)):
+        want = oracle.compact(bits(src), cu, idx, block_table=bt, page_size=ps, n_pages=n_pages)
+        want[want == 0xFFFF] = 0x7FFF                               # slots the call must not touch keep their fill
+        np.testing.assert_array_equal(bits(pool), want)
+    # a page id out of range is skipped and reported, not written
+    bad = bt.copy()
+    bad[0, 0] = n_pages
+    B.spec_compact_kv(pr, k, v, idx_t, C, kp, vp, block_table=torch.from_numpy(bad).cuda(), page_size=ps,
+                      n_pages=n_pages, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == B.ERR_BAD_ARG
+
+
+# ------------------------------------------------------------------ whole path --------
+
+def check_pipeline(B, W, oracle, w, layers, units=None):
+    """score -> pool/top-C -> gather on the GPU against the oracle; `units` restricts the oracle to
+    sampled (layer, kv head) pairs."""
+    g = Gpu(B, W, w, layers)
+    scores = g.score()
+    idx, cnt = g.topk(scores, B.POOL_MAX, w.pool_k, w.c_max)
+    ko = torch.empty((w.n_seq, g.L, w.n_kv_heads, w.c_max, w.head_dim), dtype=torch.bfloat16, device="cuda")
+    vo = torch.empty_like(ko)
+    bt = None
+    if w.page_size:
+        bt = W.block_table(w, "cuda")
+        n_pages = bt.numel()
+        ko = torch.zeros((g.L, n_pages, w.n_kv_heads, w.page_size, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        vo = torch.zeros_like(ko)
+        B.spec_compact_kv(g.pr, g.k, g.v, idx, w.c_max, ko, vo, block_table=bt, page_size=w.page_size,
+                          n_pages=n_pages, status_word=g.status)
+    else:
+        B.spec_compact_kv(g.pr, g.k, g.v, idx, w.c_max, ko, vo, status_word=g.status)
+    torch.cuda.synchronize()
+    assert g.status.item() == 0
+    G = w.group
+    units = units or [(l, h) for l in range(g.L) for h in range(w.n_kv_heads)]
+    idx_np, tot_in, tot_out = idx.cpu().numpy(), 0, 0
+    for (l, h) in units:
+        qs = g.q[:, l:l + 1, h * G:(h + 1) * G]
+        ks = g.k[l:l + 1, h:h + 1]
+        ref = oracle.spec_score(bits(qs), bits(ks), g.cu, w.n_lookahead, w.n_window, w.scale)
+        assert_scores_close(scores[l:l + 1, h:h + 1].cpu().numpy(), ref, g.cu)
+        oidx, ocnt, pooled, th = oracle.pool_topk(ref, g.cu, oracle.POOL_MAX, w.pool_k, w.c_max)
+        for s in range(w.n_seq):
+            a, b = assert_index_sets_match(idx_np[s, l, h], oidx[s, 0, 0], pooled[0, 0, g.cu[s]:g.cu[s + 1]], th[s, 0, 0])
+            tot_out += a
+            tot_in += b
+            n = g.cu[s + 1] - g.cu[s]
+            if w.planted != "token" and n >= w.c_max * 4:
+                pos = W.planted_positions(w, layers[l], s, n)[h].numpy()
+                assert set(pos).issubset(set(idx_np[s, l, h])), "planted heavy hitters must be selected"
+        # gather is bit-exact given the GPU's own indices
+        gk = oracle.compact(bits(ks), g.cu, idx_np[:, l:l + 1, h:h + 1], None if bt is None else bt.cpu().numpy(),
+                            w.page_size, 0 if bt is None else bt.numel())
+        gv = oracle.compact(bits(g.v[l:l + 1, h:h + 1]), g.cu, idx_np[:, l:l + 1, h:h + 1],
+                            None if bt is None else bt.cpu().numpy(), w.page_size, 0 if bt is None else bt.numel())
+        if bt is None:
+            np.testing.assert_array_equal(bits(ko[:, l:l + 1, h:h + 1]), gk)
+            np.testing.assert_array_equal(bits(vo[:, l:l + 1, h:h + 1]), gv)
+        else:
+            np.testing.assert_array_equal(bits(ko[l:l + 1, :, h:h + 1]), gk)
+            np.testing.assert_array_equal(bits(vo[l:l + 1, :, h:h + 1]), gv)
+    return tot_out, tot_in
+
+
+def test_pipeline_config0_full(B, W, oracle):
+    out, inside = check_pipeline(B, W, oracle, W.CONFIGS[0], [0])
+    assert out > 0
+
+
+def test_pipeline_config1_full_size_sampled_units(B, W, oracle):
+    w = W.CONFIGS[1]
+    check_pipeline(B, W, oracle, w, list(range(w.n_layers)), units=[(0, 0), (13, 5), (31, 7)])
+
+
+def test_pipeline_config2_full_size_sampled_units(B, W, oracle):
+    w = W.CONFIGS[2]
+    free, _ = torch.cuda.mem_get_info()
+    layers = list(range(w.n_layers)) if free > 40e9 else list(range(4))
+    check_pipeline(B, W, oracle, w, layers, units=[(0, 3), (len(layers) - 1, 6)])
+
+
+def test_pipeline_config4_ragged_paged_sampled_units(B, W, oracle):
+    w = W.CONFIGS[4]
+    check_pipeline(B, W, oracle, w, [0, 1], units=[(0, 2), (1, 7)])
+
+
+# ------------------------------------------------------------------ SpecPC ------------
+
+def run_keep(B, pr, scores_t, reduce, pool, k, c_max, nb, forced, cap, n_seq):
+    keep = torch.full((n_seq, cap), -7, dtype=torch.int32, device="cuda")
+    n_keep = torch.full((n_seq,), -7, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.spec_workspace_bytes(pr), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.specpc_token_select(pr, scores_t, reduce, pool, k, c_max, nb, forced, keep, cap, n_keep, ws, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    return keep.cpu().numpy(), n_keep.cpu().numpy()
+
+
+def test_specpc_exact_on_dyadic_scores(B, W, oracle):
+    """Scores on a dyadic grid sum exactly in fp32, so the keep list must equal the oracle's."""
+    rng = np.random.default_rng(6)
+    L, H = 4, 2
+    cu = [0, 900, 905, 905, 3000]
+    scores = (rng.integers(0, 64, size=(L, H, 3000)) / 64).astype(np.float32)
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda")
+    pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=64, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=3000, n_in=2095, n_seq=4, cu_seqlens=cu_t)
+    st = torch.from_numpy(scores).cuda()
+    for reduce in (0, 1):
+        for (c_max, nb, forced, k) in ((64, 8, 0, 7), (64, 0, 0, 7), (50, 3, 16, 3), (2000, 2, 0, 7), (10, 64, 4, 1)):
+            cap = 2095
+            keep, n_keep = run_keep(B, pr, st, reduce, 0, k, c_max, nb, forced, cap, 4)
+            ok, on, _, _ = oracle.specpc_select(scores.astype(np.float64), cu, reduce, 0, k, c_max, nb, forced, cap)
+            np.testing.assert_array_equal(n_keep, on)
+            np.testing.assert_array_equal(keep, ok)
+
+
+def test_specpc_config3_full(B, W, oracle):
+    w = W.CONFIGS[3]
+    g = Gpu(B, W, w, list(range(w.n_layers)))
+    scores = g.score()
+    cap = min(w.n_in, w.c_max * (2 * w.n_neighbor + 1))
+    keep, n_keep = run_keep(B, g.pr, scores, B.REDUCE_SUM, B.POOL_MAX, w.pool_k, w.c_max, w.n_neighbor, 0, cap, 1)
+    got = keep[0, :n_keep[0]]
+    assert np.all(np.diff(got) > 0) and np.all(keep[0, n_keep[0]:] == -1)
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale)
+    assert_scores_close(scores.cpu().numpy(), ref, g.cu)
+    okeep, on, tok, th = oracle.specpc_select(ref, g.cu, oracle.SUM, oracle.POOL_MAX, w.pool_k, w.c_max,
+                                              w.n_neighbor, 0, cap)
+    ref_keep = set(okeep[0, :on[0]])
+    # planted token positions and their +-8 neighbourhoods are kept
+    for p in W.planted_positions(w, 0, 0, w.n_in)[0].tolist():
+        assert set(range(max(0, p - 8), min(w.n_in - 1, p + 8) + 1)).issubset(set(got))
+    # every disagreement with the oracle is explained by a top-C candidate inside the tolerance band
+    band = 2e-3 * abs(th[0]) + 1e-6
+    near = np.flatnonzero(np.abs(tok - th[0]) <= band)
+    for j in set(got) ^ ref_keep:
+        assert np.any(np.abs(near - j) <= w.n_neighbor), "keep-list difference at %d outside the band" % j
