@@ -90,6 +90,7 @@ def make_problem(*, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: in
     p = spec_problem()
     p.n_seq = n_seq
     p.cu_seqlens = None if cu_seqlens is None else cu_seqlens.data_ptr()
+    p._keepalive = cu_seqlens            # the struct only holds the address: keep the tensor alive with it
     p.n_in = n_in
     p.total_tokens = total_tokens
     p.n_layers, p.n_q_heads, p.n_kv_heads, p.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim

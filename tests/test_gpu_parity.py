@@ -194,8 +194,11 @@ def test_compact_bit_exact_contiguous_and_paged(B, W, oracle, d):
     L, H, C = 2, 3, 70
     cu = [0, 300, 300, 1000]
     T = 1000
-    k = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
-    v = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
+    def raw():                       # arbitrary bit patterns (NaNs included), except the oracle's 0xFFFF "untouched" mark
+        a = rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)
+        a[a == -1] = 7
+        return torch.from_numpy(a).view(torch.bfloat16).cuda()
+    k, v = raw(), raw()
     idx = np.full((3, L, H, C), -1, dtype=np.int32)
     for s, n in enumerate((300, 0, 700)):
         for l in range(L):
