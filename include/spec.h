@@ -108,7 +108,8 @@ const char* spec_last_error(void);
  *  row_weight  optional device float[R], w >= 0 (Algorithm 2 lines 4-6); NULL = all ones
  *  causal_window  0: every row sees every key it is given.  1: window row r only sees keys up to
  *              its own prompt position n_s - n_window + r.
- *  scores_out  [n_layers, n_kv_heads, T] fp32; only tokens covered by cu_seqlens are written
+ *  scores_out  [n_layers, n_kv_heads, T] fp32; the whole buffer is overwritten (tokens that no
+ *              sequence covers are set to 0)
  * Limits: M*head_dim <= 81920 (e.g. M <= 640 at head_dim 128); else SPEC_ERR_UNSUPPORTED.
  */
 int32_t spec_score(const spec_problem* problem, const void* q, const void* k, const float* row_weight,

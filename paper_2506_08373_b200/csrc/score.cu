@@ -9,9 +9,14 @@
 //   pass 2   S^T = K Q^T per tile (keys on TMEM lanes, query rows on columns):
 //            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one store per key.
 // Both passes are persistent, warp-specialised kernels: warp 0 feeds K tiles (and the unit's Q)
-// with TMA into a shared-memory ring, warp 1 issues tcgen05.mma into double-buffered TMEM, warps
-// 2-5 drain TMEM with tcgen05.ld and do the exponentials.  The global key-tile space
-// (layer, KV head, sequence, tile) is cut into equal contiguous ranges, one per CTA.
+// with TMA into a shared-memory ring, warp 1 issues tcgen05.mma into four 128-column TMEM
+// buffers, and two epilogue warpgroups (warps 2-5 and 6-9) drain alternate buffers with
+// tcgen05.ld and do the exponentials, so every SM sub-partition has two epilogue warps to hide
+// the MUFU latency.  The two warpgroups never synchronise inside a unit: pass 1 writes their
+// statistics as separate partials, pass 2 adds their per-key sums into the zero-filled output
+// with one reduction each (two addends, so the result does not depend on their order).
+// The global key-tile space (layer, KV head, sequence, tile) is cut into equal contiguous
+// ranges, one per CTA.
 //
 // Every wait on an mbarrier is bounded in time; on expiry the CTA reports SPEC_ERR_TIMEOUT
 // through the status word, lets its copies land, frees its TMEM and returns.
@@ -21,7 +26,10 @@
 
 namespace spec {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kEpilogueThreads = 256;
+constexpr int kBufCols = 128;
+constexpr int kNumBufs = 4;
 constexpr int kTileKeys = 128;
 constexpr int kMaxStages = 8;
 constexpr int kMaxMTiles = 10;
@@ -31,7 +39,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 struct ScoreParams {
   const int32_t* cu;
   const float* row_weight;
-  float* partial;       // [n_units + n_ctas][M][2]  (max in log2 domain, sum-exp)
+  float* partial;       // [n_units + n_ctas][2 warpgroups][M][2]  (max in log2 domain, sum-exp)
   float* rowc;          // [n_seq*L*Hq*R]  minus the per-row constant
   float* scores;        // [L, Hkv, T]
   int32_t* status;
@@ -264,8 +272,8 @@ template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  constexpr int BUFCOLS = PASS == 1 ? 128 : 256;
-  constexpr int NBUF = 512 / BUFCOLS;
+  constexpr int BUFCOLS = kBufCols;
+  constexpr int NBUF = kNumBufs;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* k_sm = smem;
@@ -387,9 +395,10 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     }
   } else {
     // ------------------------------------------------ epilogue --------
+    const int wg = (warp - 2) >> 2;                        // warpgroup: takes the buffers with index % 2 == wg
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
-    const int et = tid - 64;                               // 0..127 among epilogue threads
+    const int et = tid - 64;                               // 0..255 among epilogue threads
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
     SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
     Seg sg;
@@ -405,6 +414,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         for (int t = 0; t < sg.nt && ok; ++t) {
           const int nv = min(kTileKeys, sg.n - (sg.t0 + t) * kTileKeys);
           for (int mt = 0; mt < n_mt; ++mt, ++bit) {
+            if ((int)(bit & 1u) != wg) continue;
             const int buf = bit % NBUF;
             ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
             if (!ok) break;
@@ -422,16 +432,16 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tmem_ld32(taddr + 96, rb);
             if (nv >= 96) stats_update<false>(ra, 32, p.a, m, z); else if (nv > 64) stats_update<true>(ra, nv - 64, p.a, m, z);
             tmem_ld_wait(rb);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&t_empty[buf]);       // all reads done: the buffer can be refilled
             if (nv >= 128) stats_update<false>(rb, 32, p.a, m, z); else if (nv > 96) stats_update<true>(rb, nv - 96, p.a, m, z);
             mrun[mt] = m;
             zrun[mt] = z;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&t_empty[buf]);
           }
         }
         if (ok) {
-          float* dst = p.partial + (size_t)(sg.unit + blockIdx.x) * p.M * 2;
+          float* dst = p.partial + ((size_t)(sg.unit + blockIdx.x) * 2 + wg) * p.M * 2;
           for (int mt = 0; mt < n_mt; ++mt) {
             const int row = mt * 128 + row_in_tile;
             if (row < p.M) {
@@ -444,13 +454,16 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     } else {
       while (ok && seg_next(it, p, tp, sg)) {
         const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
-        asm volatile("bar.sync 1, 128;" ::: "memory");          // previous unit's constants no longer read
-        for (int i = et; i < p.M_pad; i += 128) c_sm[i] = i < p.M ? p.rowc[qrow0 + i] : -INFINITY;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");          // previous unit's constants no longer read
+        for (int i = et; i < p.M_pad; i += kEpilogueThreads) c_sm[i] = i < p.M ? p.rowc[qrow0 + i] : -INFINITY;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         float* out = p.scores + ((long long)sg.l * p.Hkv + sg.h) * p.T + sg.begin;
         for (int t = 0; t < sg.nt && ok; ++t) {
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          bool mine = false;
           for (int ch = 0; ch < p.n_chunks; ++ch, ++bit) {
+            if ((int)(bit & 1u) != wg) continue;
+            mine = true;
             const int buf = bit % NBUF;
             ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
             if (!ok) break;
@@ -477,9 +490,15 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           }
           if (!ok) break;
           const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
-          if (key < sg.n) {
-            out[key] = p.reduce == SPEC_REDUCE_MAX ? fmaxf(fmaxf(acc[0], acc[1]), fmaxf(acc[2], acc[3]))
-                                                   : (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          if (mine && key < sg.n) {
+            // The output was zero-filled; each warpgroup contributes once per key.
+            if (p.reduce == SPEC_REDUCE_MAX) {
+              const float v = fmaxf(fmaxf(acc[0], acc[1]), fmaxf(acc[2], acc[3]));
+              asm volatile("red.global.max.u32 [%0], %1;" ::"l"(out + key), "r"(__float_as_uint(v)) : "memory");
+            } else {
+              const float v = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+              asm volatile("red.global.add.f32 [%0], %1;" ::"l"(out + key), "f"(v) : "memory");
+            }
           }
         }
       }
@@ -530,11 +549,12 @@ __global__ void __launch_bounds__(128) merge_kernel(const ScoreParams p, int n_c
   const int qrow0 = ((s * p.L + l) * p.Hq + h * p.G) * p.R;
   for (int i = threadIdx.x; i < p.M; i += blockDim.x) {
     float m = -INFINITY;
-    for (int c = b0; c <= b1; ++c) m = fmaxf(m, p.partial[((size_t)(unit + c) * p.M + i) * 2]);
+    const int s0 = (unit + b0) * 2, s1 = (unit + b1) * 2 + 1;       // two warpgroup partials per CTA
+    for (int c = s0; c <= s1; ++c) m = fmaxf(m, p.partial[((size_t)c * p.M + i) * 2]);
     float z = 0.f;
-    for (int c = b0; c <= b1; ++c) {
-      const float pm = p.partial[((size_t)(unit + c) * p.M + i) * 2];
-      const float pz = p.partial[((size_t)(unit + c) * p.M + i) * 2 + 1];
+    for (int c = s0; c <= s1; ++c) {
+      const float pm = p.partial[((size_t)c * p.M + i) * 2];
+      const float pz = p.partial[((size_t)c * p.M + i) * 2 + 1];
       if (pm > -INFINITY) z += pz * exp2f(pm - m);
     }
     float c = m + log2f(z);
@@ -629,7 +649,7 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   p.n_in = pr->n_in; p.n_seq = pr->n_seq; p.L = pr->n_layers; p.Hq = pr->n_q_heads; p.Hkv = pr->n_kv_heads;
   p.G = G; p.R = R; p.M = M; p.M_pad = M_pad; p.d = d;
   const int M32 = (M + 31) / 32 * 32;
-  p.n_chunks = (M32 + 255) / 256;
+  p.n_chunks = (M32 + kBufCols - 1) / kBufCols;
   p.cw = ((M32 + p.n_chunks - 1) / p.n_chunks + 31) / 32 * 32;
   p.cw_last = M32 - (p.n_chunks - 1) * p.cw;
   p.reduce = reduce;
@@ -650,6 +670,7 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
   SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  SPEC_CUDA_OK(cudaMemsetAsync(scores_out, 0, (size_t)pr->n_layers * pr->n_kv_heads * (size_t)pr->total_tokens * sizeof(float), st));
   score_kernel<1><<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
   SPEC_CUDA_OK(cudaGetLastError());
   merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);
