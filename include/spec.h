@@ -175,6 +175,36 @@ int32_t specpc_token_select(const spec_problem* problem, const float* scores, in
                             int32_t* n_keep_out, void* workspace, size_t workspace_bytes,
                             int32_t* status_word, void* stream);
 
+/*
+ * specpc_token_select for callers that cannot allocate device memory.
+ *
+ * (No counterpart in the paper: this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option -- inside an inference server
+ * whose memory pool already owns the whole device, while such a server measures its free memory,
+ * or in a plugin that only ever sees the tensors of one request.  Such a caller has no buffer to
+ * pass as `workspace`, so this variant keeps its only scratch, one fp32 token score per packed
+ * token, in an array that is part of the library itself.  The call allocates nothing and frees
+ * nothing; inputs and outputs are still the caller's.
+ *
+ * Limits and rules
+ *   - total_tokens <= SPEC_STATIC_MAX_TOKENS, else SPEC_ERR_UNSUPPORTED (the message names the
+ *     limit).  The array costs SPEC_STATIC_MAX_TOKENS * 4 bytes (1 MiB) of device memory on
+ *     every GPU that loads the library, for the life of the process.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call left there;
+ *     each call rewrites every element it later reads, so results never depend on earlier
+ *     calls -- but two calls that overlap on the GPU (different streams, no dependency) race
+ *     on it.  Order them.
+ * Arguments and results are exactly those of specpc_token_select, minus the workspace.
+ */
+#define SPEC_STATIC_MAX_TOKENS 262144
+int32_t specpc_token_select_static(const spec_problem* problem, const float* scores, int32_t layer_head_reduce,
+                                   int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,
+                                   int32_t n_forced_tail, int32_t* keep_out, int32_t keep_capacity,
+                                   int32_t* n_keep_out, int32_t* status_word, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

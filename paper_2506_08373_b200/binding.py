@@ -18,7 +18,8 @@ REDUCE_SUM, REDUCE_MAX = 0, 1
 POOL_MAX, POOL_AVG = 0, 1
 
 EXPORTS = ("spec_workspace_bytes", "spec_last_error", "spec_score", "spec_pool_topk", "spec_compact_kv",
-           "specpc_token_select")
+           "specpc_token_select", "specpc_token_select_static")
+STATIC_MAX_TOKENS = 262144
 
 
 class SpecError(RuntimeError):
@@ -64,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.spec_compact_kv.argtypes = [pp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp]
         L.specpc_token_select.restype = i32
         L.specpc_token_select.argtypes = [pp, vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, sz, vp, vp]
+        L.specpc_token_select_static.restype = i32
+        L.specpc_token_select_static.argtypes = [pp, vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -142,3 +145,13 @@ def specpc_token_select(problem, scores, layer_head_reduce, pool, pool_k, c_max,
                                      n_neighbor, n_forced_tail, _ptr(keep_out), keep_capacity, _ptr(n_keep_out),
                                      _ptr(workspace), workspace.numel() * workspace.element_size(),
                                      _ptr(status_word), _stream()))
+
+
+def specpc_token_select_static(problem, scores, layer_head_reduce, pool, pool_k, c_max, n_neighbor, n_forced_tail,
+                               keep_out, keep_capacity, n_keep_out, status_word=None):
+    """specpc_token_select without a workspace argument, for callers that cannot allocate device
+    memory: the token-score scratch is an array inside the library (at most STATIC_MAX_TOKENS
+    packed tokens).  Calls that overlap on the GPU race on that array."""
+    _check(lib().specpc_token_select_static(ctypes.byref(problem), _ptr(scores), layer_head_reduce, pool, pool_k,
+                                            c_max, n_neighbor, n_forced_tail, _ptr(keep_out), keep_capacity,
+                                            _ptr(n_keep_out), _ptr(status_word), _stream()))

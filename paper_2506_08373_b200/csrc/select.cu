@@ -443,3 +443,88 @@ SPEC_EXPORT int32_t specpc_token_select(const spec_problem* pr, const float* sco
   SPEC_CUDA_OK(cudaGetLastError());
   return SPEC_OK;
 }
+
+// ------------------------------------------------- entry point without allocations ---
+//
+// Some callers cannot hand the library a workspace because they cannot allocate device
+// memory at the point of the call: code running inside a serving engine whose allocator
+// has already claimed (or is profiling) the whole device, or a plugin that is only given
+// the tensors of the request.  For them the token-score vector of the SpecPC selection
+// lives in a fixed array that is part of the library image.
+
+namespace spec {
+
+// The scratch of specpc_token_select_static: one fp32 token score per packed token.  Every
+// device that loads the library holds these SPEC_STATIC_MAX_TOKENS * 4 bytes until the
+// process exits.  In host code this name is only a handle for cudaGetSymbolAddress; it is
+// not a device address and must never be passed to a kernel.
+static __device__ __align__(256) float g_static_token_scores[SPEC_STATIC_MAX_TOKENS];
+
+constexpr int kMaxDevices = 64;
+
+// Device address of the array on the current device, looked up once per device.
+static int static_scratch(float** out) {
+  static float* cached[kMaxDevices] = {nullptr};
+  int dev = 0;
+  SPEC_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(SPEC_ERR_UNSUPPORTED, "device ordinal %d is not supported", dev);
+  float* ptr = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
+  if (!ptr) {
+    const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_token_scores);
+    if (e != cudaSuccess || !ptr)
+      return fail(SPEC_ERR_CUDA, "cudaGetSymbolAddress(static token scratch): %s", cudaGetErrorString(e));
+    __atomic_store_n(&cached[dev], ptr, __ATOMIC_RELEASE);
+  }
+  *out = ptr;
+  return SPEC_OK;
+}
+
+}  // namespace spec
+
+SPEC_EXPORT int32_t specpc_token_select_static(const spec_problem* pr, const float* scores, int32_t layer_head_reduce,
+                                               int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,
+                                               int32_t n_forced_tail, int32_t* keep_out, int32_t keep_capacity,
+                                               int32_t* n_keep_out, int32_t* status_word, void* stream) {
+  using namespace spec;
+  int rc = check_problem(pr);
+  if (rc != SPEC_OK) return rc;
+  if (!scores || !keep_out || !n_keep_out) return fail(SPEC_ERR_BAD_ARG, "scores, keep_out and n_keep_out must not be NULL");
+  if (layer_head_reduce != SPEC_REDUCE_SUM && layer_head_reduce != SPEC_REDUCE_MAX)
+    return fail(SPEC_ERR_BAD_ARG, "layer_head_reduce=%d is not a spec_reduce value", layer_head_reduce);
+  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);
+  if (rc != SPEC_OK) return rc;
+  if (n_neighbor < 0) return fail(SPEC_ERR_BAD_ARG, "n_neighbor=%d is negative", n_neighbor);
+  if (pr->total_tokens > SPEC_STATIC_MAX_TOKENS)
+    return fail(SPEC_ERR_UNSUPPORTED, "total_tokens=%d exceeds the built-in scratch of %d tokens; use specpc_token_select with a workspace",
+                pr->total_tokens, SPEC_STATIC_MAX_TOKENS);
+  const int max_len = max_seq_len(pr);
+  const int64_t worst = (int64_t)c_max * (2 * (int64_t)n_neighbor + 1) + n_forced_tail;
+  const int64_t need_cap = worst < max_len ? worst : max_len;
+  if (keep_capacity < need_cap)
+    return fail(SPEC_ERR_BAD_ARG, "keep_capacity=%d is below the worst case %lld", keep_capacity, (long long)need_cap);
+  const int bitmap_words = (max_len + 31) / 32 + 1;
+  rc = check_device();
+  if (rc != SPEC_OK) return rc;
+  float* tok = nullptr;
+  rc = static_scratch(&tok);                 // first call on a device: looks the array's address up
+  if (rc != SPEC_OK) return rc;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t T = pr->total_tokens;
+  if (T > 0) {
+    // Writes every token score the selection reads, so nothing of an earlier call survives.
+    token_reduce_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(scores, tok, T, pr->n_layers * pr->n_kv_heads,
+                                                                     layer_head_reduce);
+    SPEC_CUDA_OK(cudaGetLastError());
+  }
+  KeepParams p;
+  p.tok = tok; p.cu = pr->cu_seqlens; p.keep_out = keep_out; p.n_keep_out = n_keep_out;
+  p.n_in = pr->n_in; p.pool = pool; p.pool_k = pool_k; p.c_max = c_max; p.n_neighbor = n_neighbor;
+  p.n_forced = n_forced_tail; p.keep_capacity = keep_capacity; p.bitmap_words = bitmap_words;
+  p.status = status_word;
+  const int smem = select_smem_bytes(max_len, bitmap_words, &p.cap);
+  SPEC_CUDA_OK(cudaFuncSetAttribute(specpc_keep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  specpc_keep_kernel<<<(unsigned)pr->n_seq, kSelThreads, smem, st>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  return SPEC_OK;
+}
