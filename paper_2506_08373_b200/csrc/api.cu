@@ -83,7 +83,7 @@ WorkspacePlan plan_workspace(const spec_problem* p) {
   w.score_ctas = (int)ctas;
   size_t off = 0;
   w.partial_off = off;
-  w.partial_bytes = (size_t)(n_units + ctas) * 2 * (size_t)M * 2 * sizeof(float);   // two epilogue warpgroups
+  w.partial_bytes = (size_t)(n_units + ctas) * 4 * (size_t)M * 2 * sizeof(float);   // four epilogue warpgroups
   off = align_up(off + w.partial_bytes, 256);
   w.rowc_off = off;
   w.rowc_bytes = (size_t)p->n_seq * p->n_layers * p->n_q_heads * (size_t)R * sizeof(float);

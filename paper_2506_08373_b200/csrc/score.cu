@@ -10,11 +10,17 @@
 //            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one store per key.
 // Both passes are persistent, warp-specialised kernels: warp 0 feeds K tiles (and the unit's Q)
 // with TMA into a shared-memory ring, warp 1 issues tcgen05.mma into four 128-column TMEM
-// buffers, and two epilogue warpgroups (warps 2-5 and 6-9) drain alternate buffers with
-// tcgen05.ld and do the exponentials, so every SM sub-partition has two epilogue warps to hide
-// the MUFU latency.  The two warpgroups never synchronise inside a unit: pass 1 writes their
-// statistics as separate partials, pass 2 adds their per-key sums into the zero-filled output
-// with one reduction each (two addends, so the result does not depend on their order).
+// buffers, and four epilogue warpgroups (16 warps, four per SM sub-partition) drain them with
+// tcgen05.ld and do the exponentials.  The warpgroups form two pairs; a pair takes a whole
+// buffer and its two warpgroups split the buffer's columns in halves, so each pair always has a
+// second buffer being filled while it works.  The exponential is the scarce resource (16 MUFU
+// results per clock per SM against 32 logits per clock from the tensor cores), so a fixed share
+// of the elements is evaluated on the FMA pipes instead (range reduction + cubic polynomial,
+// relative error 7.5e-5), and the surrounding arithmetic uses the packed two-lane fp32
+// instructions to halve its issue slots.  Warpgroups never synchronise inside a unit: pass 1
+// writes their statistics as separate partials; in pass 2 a key tile belongs to one pair, whose
+// two warpgroups add their per-key sums into the zero-filled output with one reduction each
+// (two addends, so the result does not depend on their order).
 // The global key-tile space (layer, KV head, sequence, tile) is cut into equal contiguous
 // ranges, one per CTA.
 //
@@ -26,8 +32,18 @@
 
 namespace spec {
 
-constexpr int kThreads = 320;
-constexpr int kEpilogueThreads = 256;
+constexpr int kEpilogueWarpgroups = 4;
+constexpr int kEpilogueThreads = kEpilogueWarpgroups * 128;
+constexpr int kMmaWarpB = 2 + kEpilogueThreads / 32;    // second MMA-issuing warp, after the epilogue warps
+constexpr int kThreads = 64 + kEpilogueThreads + 32;
+#ifndef SPEC_POLY_PAIRS
+#define SPEC_POLY_PAIRS 5
+#endif
+#ifndef SPEC_LOAD_AHEAD
+#define SPEC_LOAD_AHEAD 0
+#endif
+constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes
+constexpr bool kLoadAhead = SPEC_LOAD_AHEAD;  // fetch a work item's second 32 columns before the math on the first
 constexpr int kBufCols = 128;
 constexpr int kNumBufs = 4;
 constexpr int kTileKeys = 128;
@@ -35,17 +51,21 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxMTiles = 10;
 constexpr int kNumBars = 2 * kMaxStages + 2 + 8;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+#ifndef SPEC_SUSPEND_HINT_NS
+#define SPEC_SUSPEND_HINT_NS 100000
+#endif
+constexpr uint32_t kSuspendHintNs = SPEC_SUSPEND_HINT_NS;
 
 struct ScoreParams {
   const int32_t* cu;
   const float* row_weight;
-  float* partial;       // [n_units + n_ctas][2 warpgroups][M][2]  (max in log2 domain, sum-exp)
+  float* partial;       // [n_units + n_ctas][4 warpgroups][M][2]  (max in log2 domain, sum-exp)
   float* rowc;          // [n_seq*L*Hq*R]  minus the per-row constant
   float* scores;        // [L, Hkv, T]
   int32_t* status;
   long long T;
   int n_in, n_seq, L, Hq, Hkv, G, R, M, M_pad, d;
-  int n_stages, n_chunks, cw, cw_last;
+  int n_stages, n_chunks, cw_last;   // pass 2: chunks of 128 query rows, the last of cw_last (64 or 128)
   int reduce;
   float a;              // softmax_scale * log2(e)
   uint32_t q_bytes, stage_bytes;
@@ -69,22 +89,22 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Returns false when another role has given up or the time limit passed.
+// Bounded wait.  Returns false when another role has given up or the time limit passed.  The
+// suspend-time hint lets the hardware park the thread until the phase completes instead of
+// spinning in the issue slots the epilogue warps need.
 __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const uint32_t addr = smem_u32(bar);
   unsigned long long t0 = 0;
-  for (uint32_t it = 0;; ++it) {
+  for (;;) {
     uint32_t ok;
     asm volatile(
-        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
     if (ok) return true;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-    }
+    if (*abort_flag) return false;
+    const unsigned long long now = global_ns();
+    if (t0 == 0) t0 = now;
+    else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
   }
 }
 
@@ -141,16 +161,16 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // Shared-memory matrix descriptor: K-major operand, rows of 64 bf16 (128 bytes) with the
-// 128-byte swizzle TMA writes; 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                 // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
-  return d;
+// 128-byte swizzle TMA writes; 8-row groups are 1024 bytes apart.  Only the start address
+// (bits 0-13, in 16-byte units) differs between the operands of this kernel, so the issuing
+// thread keeps the low word per operand and adds offsets to it; the high word is constant.
+constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4)        // stride byte offset between 8-row groups
+                             | (1u << 14)                 // descriptor version of this architecture
+                             | (2u << 29);                // 128-byte swizzle
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) {
+  return ((saddr & 0x3FFFFu) >> 4) | (1u << 16);          // leading byte offset (unused for swizzled K-major)
 }
+__device__ __forceinline__ uint64_t desc_at(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
 __device__ __forceinline__ uint32_t make_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -216,59 +236,88 @@ __device__ bool seg_next(SegIter& it, const ScoreParams& p, const int* tp, Seg& 
 
 // ------------------------------------------------------------------ epilogue math -----
 
-// Pass 1: fold 32 logits of one row into the running (max, sum-exp), log2 domain.
-template <bool MASKED>
-__device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid, float a, float& m, float& z) {
-  float gm = -INFINITY;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const float v = __uint_as_float(r[i]);
-    if (!MASKED || i < valid) gm = fmaxf(gm, v);
-  }
-  const float mn = fmaxf(m, gm * a);
-  if (mn == -INFINITY) return;
-  const float neg = -mn;
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; i += 4) {
-    float e0 = ex2(fmaf(__uint_as_float(r[i + 0]), a, neg));
-    float e1 = ex2(fmaf(__uint_as_float(r[i + 1]), a, neg));
-    float e2 = ex2(fmaf(__uint_as_float(r[i + 2]), a, neg));
-    float e3 = ex2(fmaf(__uint_as_float(r[i + 3]), a, neg));
-    if (MASKED) {
-      if (i + 0 >= valid) e0 = 0.f;
-      if (i + 1 >= valid) e1 = 0.f;
-      if (i + 2 >= valid) e2 = 0.f;
-      if (i + 3 >= valid) e3 = 0.f;
-    }
-    s0 += e0; s1 += e1; s2 += e2; s3 += e3;
-  }
-  z = z * ex2(m - mn) + ((s0 + s1) + (s2 + s3));
-  m = mn;
+// The packed fp32 instructions (two lanes per instruction) through the float2 intrinsics.
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
-// Pass 2: probabilities of 32 query rows for this thread's key, reduced into acc[4].
+// 2^x for both lanes on the MUFU unit.
+__device__ __forceinline__ float2 ex2_mufu2(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+// 2^x for both lanes without the MUFU unit: x = n + f with n = round(x), |f| <= 1/2 (adding
+// 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic with relative error 7.5e-5,
+// then n is added into the exponent field.  x is clamped at -125 so the exponent cannot wrap.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
+  const float2 xr = __fadd2_rn(x, splat2(12582912.f));
+  const float2 n = __fadd2_rn(xr, splat2(-12582912.f));
+  const float2 f = __ffma2_rn(n, splat2(-1.f), x);
+  float2 q = __ffma2_rn(f, splat2(0.0551713221f), splat2(0.2426105440f));
+  q = __ffma2_rn(q, f, splat2(0.6932609677f));
+  q = __ffma2_rn(q, f, splat2(0.9999281168f));
+  return make_float2(__uint_as_float(__float_as_uint(q.x) + (__float_as_uint(xr.x) << 23)),
+                     __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(xr.y) << 23)));
+}
+// Pair i (0..15) of a 32-element block: kPolyPairs of them, evenly spread, avoid the MUFU unit.
+__device__ __forceinline__ constexpr bool poly_pair(int i) {
+  return (i * kPolyPairs) / 16 != ((i + 1) * kPolyPairs) / 16;
+}
+__device__ __forceinline__ float2 ex2_pair(float2 x, int i) { return poly_pair(i) ? ex2_poly2(x) : ex2_mufu2(x); }
+
+// Pass 1: fold 32 logits of one row into the running (max, sum-exp), log2 domain.  At least one
+// of the 32 logits is valid.
+template <bool MASKED>
+__device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid, float a, float& m, float& z) {
+  float v[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    v[i] = __uint_as_float(r[i]);
+    if (MASKED && i >= valid) v[i] = -INFINITY;
+  }
+  float g[11];
+#pragma unroll
+  for (int i = 0; i < 10; ++i) g[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+  g[10] = fmaxf(v[30], v[31]);
+  const float g0 = max3(g[0], g[1], g[2]), g1 = max3(g[3], g[4], g[5]), g2 = max3(g[6], g[7], g[8]);
+  const float gm = max3(max3(g0, g1, g2), g[9], g[10]);
+  const float mn = fmaxf(m, gm * a);                       // a > 0
+  z *= ex2(m - mn);                                        // first block: 0 * 2^-inf = 0
+  m = mn;
+  const float2 a2 = splat2(a), neg2 = splat2(-mn);
+  float2 s0 = splat2(0.f), s1 = splat2(0.f);
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) {
+    s0 = __fadd2_rn(s0, ex2_pair(__ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), a2, neg2), i));
+    s1 = __fadd2_rn(s1, ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1));
+  }
+  z += (s0.x + s0.y) + (s1.x + s1.y);
+}
+
+// Pass 2: probabilities of 32 query rows for this thread's key, reduced into acc (two packed
+// partial sums, or two packed maxima).
 template <bool MAXRED>
-__device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const float* __restrict__ negc, float a, float (&acc)[4]) {
+__device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const float* __restrict__ negc, float2 a2, float2 (&acc)[2]) {
   const float4* c4 = reinterpret_cast<const float4*>(negc);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const float4 c = c4[i];
-    const float p0 = ex2(fmaf(__uint_as_float(r[4 * i + 0]), a, c.x));
-    const float p1 = ex2(fmaf(__uint_as_float(r[4 * i + 1]), a, c.y));
-    const float p2 = ex2(fmaf(__uint_as_float(r[4 * i + 2]), a, c.z));
-    const float p3 = ex2(fmaf(__uint_as_float(r[4 * i + 3]), a, c.w));
+    const float2 p0 = ex2_pair(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1])), a2, make_float2(c.x, c.y)), 2 * i);
+    const float2 p1 = ex2_pair(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), a2, make_float2(c.z, c.w)), 2 * i + 1);
     if (MAXRED) {
-      acc[0] = fmaxf(acc[0], p0); acc[1] = fmaxf(acc[1], p1); acc[2] = fmaxf(acc[2], p2); acc[3] = fmaxf(acc[3], p3);
+      acc[0] = make_float2(fmaxf(acc[0].x, p0.x), fmaxf(acc[0].y, p0.y));
+      acc[1] = make_float2(fmaxf(acc[1].x, p1.x), fmaxf(acc[1].y, p1.y));
     } else {
-      acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
+      acc[0] = __fadd2_rn(acc[0], p0);
+      acc[1] = __fadd2_rn(acc[1], p1);
     }
   }
 }
 
 // ------------------------------------------------------------------ the kernel --------
 
-template <int PASS>
+template <int PASS, bool MAXRED>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -301,10 +350,11 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
   }
   if (tid == 32) {
-    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 2); }   // both MMA threads release a stage
     mbar_init(q_full, 1);
-    mbar_init(q_empty, 1);
-    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 4); }
+    mbar_init(q_empty, 2);
+    // a buffer is drained by the eight warps of one warpgroup pair
+    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -347,17 +397,25 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer ------
+  } else if (warp == 1 || warp == kMmaWarpB) {
+    // ------------------------------------------------ MMA issuers -----
+    // Two issuing threads, one per warpgroup pair.  An issuing thread is a serial chain of
+    // barrier waits and tcgen05.mma instructions (each holds the thread for about 60 cycles),
+    // so one thread alone leaves the tensor pipe idle for more than half of the time.  Thread s
+    // feeds pair s only and owns that pair's two TMEM buffers (s and s + 2).  Both threads
+    // wait for every key tile and commit to its "empty" barrier, whether or not they used it,
+    // so that every phase of those barriers sees exactly two arrivals.
     if (lane == 0) {
+      const int strm = warp == 1 ? 0 : 1;
       SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
       Seg sg;
-      uint32_t kit = 0, bit = 0, nseg = 0;
+      uint32_t kit = 0, bit = 0, nseg = 0, j = 0;            // j: items issued to my pair
       bool ok = true;
-      const uint32_t idesc_full = make_idesc(PASS == 1 ? 128 : p.cw);
+      const uint32_t idesc_full = make_idesc(128);
       const uint32_t idesc_last = make_idesc(PASS == 1 ? 128 : p.cw_last);
       const int n_sub = PASS == 1 ? p.M_pad / 128 : p.n_chunks;
-      const uint32_t q_base = smem_u32(q_sm);
+      const uint32_t q_lo0 = desc_lo(smem_u32(q_sm)), k_lo0 = desc_lo(smem_u32(k_sm));
+      const uint32_t q_half16 = q_half_bytes >> 4;
       while (ok && seg_next(it, p, tp, sg)) {
         ok = mbar_wait(q_full, nseg & 1, abort_flag);
         if (!ok) break;
@@ -368,37 +426,51 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t k_base = smem_u32(k_sm + (size_t)stage * p.stage_bytes);
-          for (int sub = 0; sub < n_sub; ++sub, ++bit) {
-            const int buf = bit % NBUF;
-            ok = mbar_wait(&t_empty[buf], ((bit / NBUF) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
-            const uint32_t q_off = PASS == 1 ? sub * (128 * 128) : sub * p.cw * 128;
-            const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
-            for (int kh = 0; kh < n_kh; ++kh) {
+          const uint32_t k_lo = k_lo0 + stage * (p.stage_bytes >> 4);
+          // Pass 1: the tile's blocks of 128 query rows alternate between the pairs (item b of
+          // the CTA goes to pair b % 2).  Pass 2: the whole tile, all chunks of query rows,
+          // belongs to the pair with the parity of the tile's index in the segment, so that a
+          // key is reduced by one pair only.
+          const bool whole_tile_mine = PASS == 2 && (t & 1) == strm;
+          if (PASS == 1 || whole_tile_mine) {
+            for (int sub = 0; sub < n_sub; ++sub, ++bit) {
+              if (PASS == 1 && (int)(bit & 1u) != strm) continue;
+              const int buf = strm + 2 * (int)(j & 1u);
+              ok = mbar_wait(&t_empty[buf], ((j >> 1) & 1) ^ 1, abort_flag);
+              if (!ok) break;
+              ++j;
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
+              const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);      // 128 query rows of 128 bytes
+              const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks) {
-                const uint64_t qd = make_desc(q_base + kh * q_half_bytes + q_off + ks * 32);
-                const uint64_t kd = make_desc(k_base + kh * (128 * 128) + ks * 32);
-                if (PASS == 1) tc_mma(d_tmem, qd, kd, idesc, (kh | ks) != 0);
-                else           tc_mma(d_tmem, kd, qd, idesc, (kh | ks) != 0);
+              for (int kh = 0; kh < 2; ++kh) {
+                if (kh < n_kh) {
+#pragma unroll
+                  for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t qd = desc_at(q_lo + kh * q_half16 + ks * 2);
+                    const uint64_t kd = desc_at(k_lo + kh * ((128 * 128) >> 4) + ks * 2);
+                    if (PASS == 1) tc_mma(d_tmem, qd, kd, idesc, (kh | ks) != 0);
+                    else           tc_mma(d_tmem, kd, qd, idesc, (kh | ks) != 0);
+                  }
+                }
               }
+              tc_commit(&t_full[buf]);
             }
-            tc_commit(&t_full[buf]);
           }
-          if (ok) tc_commit(&k_empty[stage]);      // stage reusable once these MMAs retire
+          if (ok) tc_commit(&k_empty[stage]);        // arrives once my MMAs on this stage (if any) retire
         }
         if (ok) tc_commit(q_empty);
       }
     }
-  } else {
+  } else if (warp < kMmaWarpB) {
     // ------------------------------------------------ epilogue --------
-    const int wg = (warp - 2) >> 2;                        // warpgroup: takes the buffers with index % 2 == wg
+    const int wg = (warp - 2) >> 2;                        // warpgroup 0..3
+    const int pair = wg >> 1;                              // pairs take alternate work items
+    const int half = wg & 1;                               // column half of the pair's buffer
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
-    const int et = tid - 64;                               // 0..255 among epilogue threads
+    const int et = tid - 64;                               // 0..511 among epilogue threads
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
     SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
     Seg sg;
@@ -406,42 +478,53 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     bool ok = true;
     uint32_t ra[32], rb[32];
     if (PASS == 1) {
+      // Work item = one 128 x 128 logit tile (query rows on lanes); this warpgroup owns 64 of
+      // its key columns.
       const int n_mt = p.M_pad / 128;
       float mrun[kMaxMTiles], zrun[kMaxMTiles];
       while (ok && seg_next(it, p, tp, sg)) {
 #pragma unroll
         for (int i = 0; i < kMaxMTiles; ++i) { mrun[i] = -INFINITY; zrun[i] = 0.f; }
         for (int t = 0; t < sg.nt && ok; ++t) {
-          const int nv = min(kTileKeys, sg.n - (sg.t0 + t) * kTileKeys);
+          const int nvh = min(kTileKeys, sg.n - (sg.t0 + t) * kTileKeys) - half * 64;   // valid keys in my half
           for (int mt = 0; mt < n_mt; ++mt, ++bit) {
-            if ((int)(bit & 1u) != wg) continue;
+            if ((int)(bit & 1u) != pair) continue;
             const int buf = bit % NBUF;
             ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = lane_base + buf * BUFCOLS;
             float m = mrun[mt], z = zrun[mt];
-            tmem_ld32(taddr, ra);
-            tmem_ld_wait(ra);
-            tmem_ld32(taddr + 32, rb);
-            if (nv >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nv, p.a, m, z);
-            tmem_ld_wait(rb);
-            tmem_ld32(taddr + 64, ra);
-            if (nv >= 64) stats_update<false>(rb, 32, p.a, m, z); else if (nv > 32) stats_update<true>(rb, nv - 32, p.a, m, z);
-            tmem_ld_wait(ra);
-            tmem_ld32(taddr + 96, rb);
-            if (nv >= 96) stats_update<false>(ra, 32, p.a, m, z); else if (nv > 64) stats_update<true>(ra, nv - 64, p.a, m, z);
-            tmem_ld_wait(rb);
+            if (nvh > 0) {
+              const uint32_t taddr = lane_base + buf * BUFCOLS + half * 64;
+              tmem_ld32(taddr, ra);
+              if (kLoadAhead) {
+                if (nvh > 32) tmem_ld32(taddr + 32, rb);
+                tmem_ld_wait(ra);
+                if (nvh > 32) tmem_ld_wait(rb);
+              } else {
+                tmem_ld_wait(ra);
+                if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z);
+                if (nvh > 32) {
+                  tmem_ld32(taddr + 32, ra);
+                  tmem_ld_wait(ra);
+                }
+              }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);       // all reads done: the buffer can be refilled
-            if (nv >= 128) stats_update<false>(rb, 32, p.a, m, z); else if (nv > 96) stats_update<true>(rb, nv - 96, p.a, m, z);
+            if (kLoadAhead) {
+              if (nvh > 0) { if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z); }
+              if (nvh >= 64) stats_update<false>(rb, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(rb, nvh - 32, p.a, m, z);
+            } else {
+              if (nvh >= 64) stats_update<false>(ra, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(ra, nvh - 32, p.a, m, z);
+            }
             mrun[mt] = m;
             zrun[mt] = z;
           }
         }
         if (ok) {
-          float* dst = p.partial + ((size_t)(sg.unit + blockIdx.x) * 2 + wg) * p.M * 2;
+          float* dst = p.partial + ((size_t)(sg.unit + blockIdx.x) * kEpilogueWarpgroups + wg) * p.M * 2;
           for (int mt = 0; mt < n_mt; ++mt) {
             const int row = mt * 128 + row_in_tile;
             if (row < p.M) {
@@ -452,51 +535,61 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
       }
     } else {
-      while (ok && seg_next(it, p, tp, sg)) {
+      // Work item = one key tile (keys on lanes) with all its chunks of 128 query rows; this
+      // warpgroup owns half of every chunk's columns.
+      const float2 a2 = splat2(p.a);
+      uint32_t j = 0;                                        // this pair's item counter
+      // Every epilogue thread passes the two barriers of every segment, also after a wait has
+      // given up, so that no warp is left waiting at them.
+      while (seg_next(it, p, tp, sg)) {
         const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
-        asm volatile("bar.sync 1, 256;" ::: "memory");          // previous unit's constants no longer read
+        asm volatile("bar.sync 1, 512;" ::: "memory");          // previous unit's constants no longer read
         for (int i = et; i < p.M_pad; i += kEpilogueThreads) c_sm[i] = i < p.M ? p.rowc[qrow0 + i] : -INFINITY;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         float* out = p.scores + ((long long)sg.l * p.Hkv + sg.h) * p.T + sg.begin;
-        for (int t = 0; t < sg.nt && ok; ++t) {
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          bool mine = false;
-          for (int ch = 0; ch < p.n_chunks; ++ch, ++bit) {
-            if ((int)(bit & 1u) != wg) continue;
-            mine = true;
-            const int buf = bit % NBUF;
-            ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
+        for (int t = pair; t < sg.nt && ok; t += 2) {
+          float2 acc[2] = {splat2(0.f), splat2(0.f)};
+          for (int ch = 0; ch < p.n_chunks; ++ch, ++j) {
+            const int buf = pair + 2 * (int)(j & 1u);
+            ok = mbar_wait(&t_full[buf], (j >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = lane_base + buf * BUFCOLS;
-            const int ng = (ch == p.n_chunks - 1 ? p.cw_last : p.cw) / 32;
-            const float* negc = c_sm + ch * p.cw;
+            const int hw = (ch == p.n_chunks - 1 ? p.cw_last : 128) >> 1;     // my columns: 32 or 64
+            const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
+            const float* negc = c_sm + ch * 128 + half * hw;
             tmem_ld32(taddr, ra);
-            for (int g = 0; g < ng; g += 2) {
+            if (kLoadAhead) {
+              if (hw > 32) tmem_ld32(taddr + 32, rb);
               tmem_ld_wait(ra);
-              if (g + 1 < ng) tmem_ld32(taddr + (g + 1) * 32, rb);
-              if (p.reduce == SPEC_REDUCE_MAX) prob_accumulate<true>(ra, negc + g * 32, p.a, acc);
-              else                             prob_accumulate<false>(ra, negc + g * 32, p.a, acc);
-              if (g + 1 < ng) {
-                tmem_ld_wait(rb);
-                if (g + 2 < ng) tmem_ld32(taddr + (g + 2) * 32, ra);
-                if (p.reduce == SPEC_REDUCE_MAX) prob_accumulate<true>(rb, negc + (g + 1) * 32, p.a, acc);
-                else                             prob_accumulate<false>(rb, negc + (g + 1) * 32, p.a, acc);
+              if (hw > 32) tmem_ld_wait(rb);
+            } else {
+              tmem_ld_wait(ra);
+              if (hw > 32) {
+                prob_accumulate<MAXRED>(ra, negc, a2, acc);
+                tmem_ld32(taddr + 32, ra);
+                tmem_ld_wait(ra);
               }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);
+            if (kLoadAhead) {
+              prob_accumulate<MAXRED>(ra, negc, a2, acc);
+              if (hw > 32) prob_accumulate<MAXRED>(rb, negc + 32, a2, acc);
+            } else {
+              prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
+            }
           }
           if (!ok) break;
           const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
-          if (mine && key < sg.n) {
-            // The output was zero-filled; each warpgroup contributes once per key.
-            if (p.reduce == SPEC_REDUCE_MAX) {
-              const float v = fmaxf(fmaxf(acc[0], acc[1]), fmaxf(acc[2], acc[3]));
+          if (key < sg.n) {
+            // The output was zero-filled; the two warpgroups of the pair contribute once per key.
+            const float v0 = acc[0].x, v1 = acc[0].y, v2 = acc[1].x, v3 = acc[1].y;
+            if (MAXRED) {
+              const float v = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
               asm volatile("red.global.max.u32 [%0], %1;" ::"l"(out + key), "r"(__float_as_uint(v)) : "memory");
             } else {
-              const float v = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+              const float v = (v0 + v1) + (v2 + v3);
               asm volatile("red.global.add.f32 [%0], %1;" ::"l"(out + key), "f"(v) : "memory");
             }
           }
@@ -549,7 +642,7 @@ __global__ void __launch_bounds__(128) merge_kernel(const ScoreParams p, int n_c
   const int qrow0 = ((s * p.L + l) * p.Hq + h * p.G) * p.R;
   for (int i = threadIdx.x; i < p.M; i += blockDim.x) {
     float m = -INFINITY;
-    const int s0 = (unit + b0) * 2, s1 = (unit + b1) * 2 + 1;       // two warpgroup partials per CTA
+    const int s0 = (unit + b0) * kEpilogueWarpgroups, s1 = (unit + b1) * kEpilogueWarpgroups + kEpilogueWarpgroups - 1;   // one partial per warpgroup and CTA
     for (int c = s0; c <= s1; ++c) m = fmaxf(m, p.partial[((size_t)c * p.M + i) * 2]);
     float z = 0.f;
     for (int c = s0; c <= s1; ++c) {
@@ -648,10 +741,9 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   p.T = pr->total_tokens;
   p.n_in = pr->n_in; p.n_seq = pr->n_seq; p.L = pr->n_layers; p.Hq = pr->n_q_heads; p.Hkv = pr->n_kv_heads;
   p.G = G; p.R = R; p.M = M; p.M_pad = M_pad; p.d = d;
-  const int M32 = (M + 31) / 32 * 32;
-  p.n_chunks = (M32 + kBufCols - 1) / kBufCols;
-  p.cw = ((M32 + p.n_chunks - 1) / p.n_chunks + 31) / 32 * 32;
-  p.cw_last = M32 - (p.n_chunks - 1) * p.cw;
+  const int M64 = (M + 63) / 64 * 64;                      // pass 2 splits each chunk's columns in two halves of 32 or 64
+  p.n_chunks = (M64 + 127) / 128;
+  p.cw_last = M64 - (p.n_chunks - 1) * 128;
   p.reduce = reduce;
   p.a = (float)((double)pr->softmax_scale * 1.4426950408889634);
   p.q_bytes = (uint32_t)M_pad * d * 2;
@@ -668,14 +760,16 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int n_ctas = wp.score_ctas;
   const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
-  SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  auto pass1 = score_kernel<1, false>;
+  auto pass2 = reduce == SPEC_REDUCE_MAX ? score_kernel<2, true> : score_kernel<2, false>;
+  SPEC_CUDA_OK(cudaFuncSetAttribute(pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  SPEC_CUDA_OK(cudaFuncSetAttribute(pass2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   SPEC_CUDA_OK(cudaMemsetAsync(scores_out, 0, (size_t)pr->n_layers * pr->n_kv_heads * (size_t)pr->total_tokens * sizeof(float), st));
-  score_kernel<1><<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+  pass1<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
   SPEC_CUDA_OK(cudaGetLastError());
   merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);
   SPEC_CUDA_OK(cudaGetLastError());
-  score_kernel<2><<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+  pass2<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
   SPEC_CUDA_OK(cudaGetLastError());
   return SPEC_OK;
 }
