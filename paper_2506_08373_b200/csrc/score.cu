@@ -37,7 +37,7 @@ constexpr int kEpilogueThreads = kEpilogueWarpgroups * 128;
 constexpr int kMmaWarpB = 2 + kEpilogueThreads / 32;    // second MMA-issuing warp, after the epilogue warps
 constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_POLY_PAIRS
-#define SPEC_POLY_PAIRS 5
+#define SPEC_POLY_PAIRS 3
 #endif
 #ifndef SPEC_LOAD_AHEAD
 #define SPEC_LOAD_AHEAD 0

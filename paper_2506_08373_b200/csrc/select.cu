@@ -188,12 +188,164 @@ struct TopkParams {
   int n_in, L, H, pool, pool_k, c_max, n_forced, cap;
 };
 
-__global__ void __launch_bounds__(kSelThreads) pool_topk_kernel(TopkParams p) {
+// ------------------------------------------------------ streaming pool + top-C ------
+//
+// One CTA per (sequence, layer, KV head) unit, any length.  The unit's scores are streamed
+// twice in chunks of kChunk positions through a two-stage cp.async ring:
+//   sweep A  pooled keys -> histogram of their top kTopBits bits (shared-memory atomics,
+//            equal neighbours aggregated); the bin holding the C-th largest key is located;
+//   sweep B  (served by L2) every key in or above that bin is appended, in position order,
+//            to a candidate list in shared memory;
+// the remaining bits are then resolved by radix passes over the candidates only, and the
+// winners are written in ascending position.  Units with at most kCandCap positions skip
+// sweep A.  If the candidates do not fit (many nearly equal scores), the unit falls back to
+// the generic multi-pass selection that recomputes keys from global memory.
+constexpr int kChunk = 4096;                      // positions per chunk: 8 consecutive per thread
+constexpr int kPerThread = kChunk / kSelThreads;
+constexpr int kTopBits = 13;
+constexpr int kTopBins = 1 << kTopBits;
+constexpr int kCandCap = 8192;
+constexpr int kStageFloats = kChunk + 256;        // chunk + halo (pool_k <= 255), a multiple of 16 bytes
+constexpr int kFinBins = 1024;                    // histogram of the candidate passes (10 bits)
+
+// Block-wide exclusive scan of one int per thread; total returned to every thread.
+// wsum: kSelWarps + 1 ints of shared memory.  Contains two __syncthreads.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) wsum[warp] = incl;
+  __syncthreads();
+  int before = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kSelWarps; ++w) {
+    const int x = wsum[w];
+    if (w < warp) before += x;
+    tot += x;
+  }
+  __syncthreads();
+  total = tot;
+  return before + incl - v;
+}
+
+// Issues the asynchronous copy of chunk `c` (positions [c*kChunk - h_lo, c*kChunk + kChunk +
+// h_hi)) of the eligible range [0, e) into `stage`; positions outside the range get `fill`.
+__device__ __forceinline__ void chunk_load(float* stage, const float* __restrict__ src, int e, int c, int h_lo, int span,
+                                           float fill) {
+  const int first = c * kChunk - h_lo;
+  for (int i = threadIdx.x; i < span; i += kSelThreads) {
+    const int j = first + i;
+    if (j >= 0 && j < e) {
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(stage + i)), "l"(src + j) : "memory");
+    } else {
+      stage[i] = fill;
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// Pooled keys of this thread's kPerThread consecutive positions of the staged chunk.
+// stage[i] holds the score of position chunk_begin - h_lo + i (or the fill value).
+template <bool MAX7>
+__device__ __forceinline__ void chunk_keys(const float* stage, int pool, int k, uint32_t (&key)[kPerThread]) {
+  const int o = threadIdx.x * kPerThread;
+  if (MAX7) {
+    float w[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 v = *reinterpret_cast<const float4*>(stage + o + 4 * i);
+      w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      const float a = fmaxf(fmaxf(w[u], w[u + 1]), fmaxf(w[u + 2], w[u + 3]));
+      const float b = fmaxf(fmaxf(w[u + 4], w[u + 5]), w[u + 6]);
+      key[u] = to_key(fmaxf(a, b));
+    }
+  } else {
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      const float* wdw = stage + o + u;
+      float acc;
+      if (pool == SPEC_POOL_MAX) {
+        acc = wdw[0];
+        for (int t = 1; t < k; ++t) acc = fmaxf(acc, wdw[t]);
+      } else {
+        acc = 0.f;
+        for (int t = 0; t < k; ++t) acc += wdw[t];
+        acc = acc / (float)k;
+      }
+      key[u] = to_key(acc);
+    }
+  }
+}
+
+// Streams the pooled keys of the eligible range [0, e) chunk by chunk; f(key, j0) receives the
+// keys of positions j0 .. j0 + kPerThread - 1 (positions >= e carry no meaning).  f is called
+// by every thread the same number of times and may synchronise the CTA.
+template <class F>
+__device__ __forceinline__ void sweep(const float* __restrict__ src, int e, int pool, int k, float* stages, F f) {
+  const int h_lo = k >> 1, span = kChunk + k - 1;
+  const float fill = pool == SPEC_POOL_MAX ? -INFINITY : 0.f;
+  const int n_chunks = (e + kChunk - 1) / kChunk;
+  const bool max7 = pool == SPEC_POOL_MAX && k == 7;
+  chunk_load(stages, src, e, 0, h_lo, span, fill);
+  for (int c = 0; c < n_chunks; ++c) {
+    float* stage = stages + (c & 1) * kStageFloats;
+    if (c + 1 < n_chunks) {
+      chunk_load(stages + ((c + 1) & 1) * kStageFloats, src, e, c + 1, h_lo, span, fill);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t key[kPerThread];
+    if (max7) chunk_keys<true>(stage, pool, k, key); else chunk_keys<false>(stage, pool, k, key);
+    f(key, c * kChunk + (int)threadIdx.x * kPerThread);
+    __syncthreads();                                       // the stage may be refilled
+  }
+}
+
+// Finds the bin holding the need-th largest element of a histogram whose bins are spread
+// over the threads, bins_per_thread consecutive bins each (need >= 1, need <= total count).
+// Returns the bin and the number of elements in higher bins to every thread.
+__device__ __forceinline__ void locate_bin(const uint32_t* hist, int bins_per_thread, int need, int* wsum, int* out2,
+                                           int& bin, int& above) {
+  const int b0 = threadIdx.x * bins_per_thread;
+  int mine = 0;
+  for (int i = 0; i < bins_per_thread; ++i) mine += (int)hist[b0 + i];
+  int total;
+  const int below = block_exclusive_scan(mine, wsum, total);
+  const int over = total - below - mine;                   // elements in bins above my range
+  if (over < need && need <= over + mine) {
+    int cum = over, b = bins_per_thread - 1;
+    for (; b > 0; --b) {
+      const int hcount = (int)hist[b0 + b];
+      if (cum + hcount >= need) break;
+      cum += hcount;
+    }
+    out2[0] = b0 + b;
+    out2[1] = cum;
+  }
+  __syncthreads();
+  bin = out2[0];
+  above = out2[1];
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  SelectScratch sc;
-  sc.hist = reinterpret_cast<uint32_t*>(smem_raw);
-  sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
-  uint32_t* keys = reinterpret_cast<uint32_t*>(sc.misc + 2 * kSelWarps + 8);
+  uint32_t* top_hist = reinterpret_cast<uint32_t*>(smem_raw);            // sweep A; later the candidate keys
+  uint32_t* cand_key = top_hist;
+  int32_t* cand_idx = reinterpret_cast<int32_t*>(top_hist + kTopBins);
+  float* stages = reinterpret_cast<float*>(cand_idx + kCandCap);
+  int* wsum = reinterpret_cast<int*>(stages + 2 * kStageFloats);        // kSelWarps + 1 (+ 2 results)
+  int* out2 = wsum + kSelWarps + 1;
+  uint32_t* fin_hist = reinterpret_cast<uint32_t*>(stages);             // candidate passes, after the sweeps
 
   const int unit = blockIdx.x;
   const int h = unit % p.H, l = (unit / p.H) % p.L, s = unit / (p.H * p.L);
@@ -204,27 +356,118 @@ __global__ void __launch_bounds__(kSelThreads) pool_topk_kernel(TopkParams p) {
   const int take = min(p.c_max - forced, e);
   int32_t* idx = p.idx_out + (int64_t)unit * p.c_max;
   const int tid = threadIdx.x;
+  const float* src = p.scores + ((int64_t)l * p.H + h) * p.T + begin;
 
   if (take > 0 && take < e) {
-    KeySource key;
-    key.scores = p.scores + ((int64_t)l * p.H + h) * p.T + begin;
-    key.e = e; key.pool = p.pool; key.k = p.pool_k;
-    key.keys = nullptr;
-    if (e <= p.cap) {
-      for (int j = tid; j < e; j += kSelThreads) keys[j] = key(j);
-      key.keys = keys;
+    // ---- sweep A: which bin of the top kTopBits bits holds the take-th largest key
+    int b1 = 0, above = 0;
+    bool fits = true;
+    if (e > kCandCap) {
+      for (int i = tid; i < kTopBins; i += kSelThreads) top_hist[i] = 0;
       __syncthreads();
+      sweep(src, e, p.pool, p.pool_k, stages, [&](const uint32_t (&key)[kPerThread], int j0) {
+        uint32_t run_d = 0xffffffffu, run_c = 0;
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) {
+          if (j0 + u < e) {
+            const uint32_t dg = key[u] >> (32 - kTopBits);
+            if (dg == run_d) {
+              ++run_c;
+            } else {
+              if (run_c) atomicAdd(&top_hist[run_d], run_c);
+              run_d = dg;
+              run_c = 1;
+            }
+          }
+        }
+        if (run_c) atomicAdd(&top_hist[run_d], run_c);
+      });
+      locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, b1, above);
+      fits = above + (int)top_hist[b1] <= kCandCap;
+      __syncthreads();                                     // top_hist is dead: its memory becomes cand_key
     }
-    uint32_t T;
-    int need_eq;
-    radix_select(key, e, take, sc, T, need_eq);
-    ordered_emit(key, e, T, need_eq, sc, [&](int rank, int j) { idx[rank] = j; });
+    if (fits) {
+      // ---- sweep B: candidates (keys in or above bin b1) in position order
+      int n_cand = 0;
+      sweep(src, e, p.pool, p.pool_k, stages, [&](const uint32_t (&key)[kPerThread], int j0) {
+        int cnt = 0;
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) cnt += (j0 + u < e) && (int)(key[u] >> (32 - kTopBits)) >= b1;
+        int total;
+        int at = n_cand + block_exclusive_scan(cnt, wsum, total);
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) {
+          if ((j0 + u < e) && (int)(key[u] >> (32 - kTopBits)) >= b1) {
+            cand_key[at] = key[u];
+            cand_idx[at] = j0 + u;
+            ++at;
+          }
+        }
+        n_cand += total;
+      });
+      // ---- remaining bits on the candidates only
+      int known = e > kCandCap ? kTopBits : 0;
+      uint32_t prefix = e > kCandCap ? (uint32_t)b1 << (32 - kTopBits) : 0u;
+      uint32_t mask = e > kCandCap ? ~((1u << (32 - kTopBits)) - 1u) : 0u;
+      int remaining = take - above;
+      while (known < 32) {
+        const int w = min(10, 32 - known), shift = 32 - known - w;
+        for (int i = tid; i < kFinBins; i += kSelThreads) fin_hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < n_cand; i += kSelThreads) {
+          const uint32_t kk = cand_key[i];
+          if ((kk & mask) == prefix) atomicAdd(&fin_hist[(kk >> shift) & ((1u << w) - 1u)], 1u);
+        }
+        __syncthreads();
+        int dg, ab;
+        locate_bin(fin_hist, kFinBins / kSelThreads, remaining, wsum, out2, dg, ab);
+        remaining -= ab;
+        prefix |= (uint32_t)dg << shift;
+        mask |= ((1u << w) - 1u) << shift;
+        known += w;
+      }
+      // ---- ordered emission: key > T, or key == T among the first `remaining` equal keys
+      const uint32_t T = prefix;
+      const int need_eq = remaining;
+      const int per = (n_cand + kSelThreads - 1) / kSelThreads;
+      const int i0 = min(tid * per, n_cand), i1 = min(i0 + per, n_cand);
+      int gt = 0, eq = 0;
+      for (int i = i0; i < i1; ++i) { const uint32_t kk = cand_key[i]; gt += kk > T; eq += kk == T; }
+      int total;
+      const int packed = block_exclusive_scan(gt | (eq << 16), wsum, total);   // n_cand <= 8192 < 2^16
+      int pre_gt = packed & 0xffff, pre_eq = packed >> 16;
+      for (int i = i0; i < i1; ++i) {
+        const uint32_t kk = cand_key[i];
+        if (kk > T) {
+          idx[pre_gt + min(pre_eq, need_eq)] = cand_idx[i];
+          ++pre_gt;
+        } else if (kk == T) {
+          if (pre_eq < need_eq) idx[pre_gt + pre_eq] = cand_idx[i];
+          ++pre_eq;
+        }
+      }
+    } else {
+      // ---- too many keys share the leading bits: generic selection, keys recomputed per pass
+      SelectScratch sc;
+      sc.hist = reinterpret_cast<uint32_t*>(stages);
+      sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
+      KeySource key;
+      key.scores = src;
+      key.e = e; key.pool = p.pool; key.k = p.pool_k;
+      key.keys = nullptr;
+      uint32_t T;
+      int need_eq;
+      radix_select(key, e, take, sc, T, need_eq);
+      ordered_emit(key, e, T, need_eq, sc, [&](int rank, int j) { idx[rank] = j; });
+    }
   } else {
     for (int c = tid; c < take; c += kSelThreads) idx[c] = c;      // every eligible position is kept
   }
   for (int c = take + tid; c < p.c_max; c += kSelThreads) idx[c] = (c - take < forced) ? e + (c - take) : -1;
   if (p.count_out && tid == 0) p.count_out[unit] = take + forced;
 }
+
+constexpr int kTopkSmemBytes = kTopBins * 4 + kCandCap * 4 + 2 * kStageFloats * 4 + (kSelWarps + 1 + 2) * 4 + 16;
 
 // ---------------------------------------------------------------------- SpecPC ------
 
@@ -388,7 +631,8 @@ SPEC_EXPORT int32_t spec_pool_topk(const spec_problem* pr, const float* scores, 
   p.scores = scores; p.cu = pr->cu_seqlens; p.idx_out = idx_out; p.count_out = count_out;
   p.T = pr->total_tokens; p.n_in = pr->n_in; p.L = pr->n_layers; p.H = pr->n_kv_heads;
   p.pool = pool; p.pool_k = pool_k; p.c_max = c_max; p.n_forced = n_forced_tail;
-  const int smem = select_smem_bytes(max_seq_len(pr), 0, &p.cap);
+  p.cap = 0;
+  const int smem = kTopkSmemBytes;
   SPEC_CUDA_OK(cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
   pool_topk_kernel<<<n_units, kSelThreads, smem, static_cast<cudaStream_t>(stream)>>>(p);
