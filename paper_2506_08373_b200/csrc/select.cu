@@ -20,7 +20,7 @@ constexpr int kSmemLimit = 227 * 1024;
 // Monotone map float -> uint32 (larger float <=> larger key), valid for any sign.
 __device__ __forceinline__ uint32_t to_key(float v) {
   const uint32_t b = __float_as_uint(v);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);   // negative: all bits flipped; else: sign bit set
 }
 
 // Pooled value of position j over the eligible range [0, e).
@@ -191,25 +191,26 @@ struct TopkParams {
 // ------------------------------------------------------ streaming pool + top-C ------
 //
 // One CTA per (sequence, layer, KV head) unit, any length.  The unit's scores are streamed
-// twice in chunks of kChunk positions through a two-stage cp.async ring:
-//   sweep A  pooled keys -> histogram of their top kTopBits bits (shared-memory atomics,
-//            equal neighbours aggregated); the bin holding the C-th largest key is located;
+// twice, kChunk positions per step, straight from global memory into registers (16-byte
+// loads, the next step's loads in flight while the current one is processed):
+//   sweep A  pooled keys -> histogram of their top kTopBits bits (shared-memory atomics);
+//            the bin holding the C-th largest key is located;
 //   sweep B  (served by L2) every key in or above that bin is appended, in position order,
 //            to a candidate list in shared memory;
 // the remaining bits are then resolved by radix passes over the candidates only, and the
 // winners are written in ascending position.  Units with at most kCandCap positions skip
 // sweep A.  If the candidates do not fit (many nearly equal scores), the unit falls back to
 // the generic multi-pass selection that recomputes keys from global memory.
-constexpr int kChunk = 4096;                      // positions per chunk: 8 consecutive per thread
+constexpr int kChunk = 4096;                      // positions per step: 8 consecutive per thread
 constexpr int kPerThread = kChunk / kSelThreads;
 constexpr int kTopBits = 13;
 constexpr int kTopBins = 1 << kTopBits;
 constexpr int kCandCap = 8192;
-constexpr int kStageFloats = kChunk + 256;        // chunk + halo (pool_k <= 255), a multiple of 16 bytes
 constexpr int kFinBins = 1024;                    // histogram of the candidate passes (10 bits)
 
 // Block-wide exclusive scan of one int per thread; total returned to every thread.
-// wsum: kSelWarps + 1 ints of shared memory.  Contains two __syncthreads.
+// wsum: kSelWarps ints of shared memory that no thread touches again before the CTA's next
+// synchronisation after this call (callers alternate two buffers).  One __syncthreads.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int& total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int incl = v;
@@ -220,102 +221,110 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int& total
   }
   if (lane == 31) wsum[warp] = incl;
   __syncthreads();
-  int before = 0, tot = 0;
+  // every warp scans the kSelWarps (<= 32) warp totals itself
+  int ws = lane < kSelWarps ? wsum[lane] : 0;
+  int wincl = ws;
 #pragma unroll
-  for (int w = 0; w < kSelWarps; ++w) {
-    const int x = wsum[w];
-    if (w < warp) before += x;
-    tot += x;
+  for (int o = 1; o < kSelWarps; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, wincl, o);
+    if (lane >= o) wincl += t;
   }
-  __syncthreads();
-  total = tot;
+  total = __shfl_sync(0xffffffffu, wincl, kSelWarps - 1);
+  const int before = __shfl_sync(0xffffffffu, wincl - ws, warp);
   return before + incl - v;
 }
 
-// Issues the asynchronous copy of chunk `c` (positions [c*kChunk - h_lo, c*kChunk + kChunk +
-// h_hi)) of the eligible range [0, e) into `stage`; positions outside the range get `fill`.
-__device__ __forceinline__ void chunk_load(float* stage, const float* __restrict__ src, int e, int c, int h_lo, int span,
-                                           float fill) {
-  const int first = c * kChunk - h_lo;
-  for (int i = threadIdx.x; i < span; i += kSelThreads) {
-    const int j = first + i;
-    if (j >= 0 && j < e) {
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(stage + i)), "l"(src + j) : "memory");
+// Geometry of the sweeps.  Positions are shifted by the unit's misalignment `mis` (0..3
+// elements from a 16-byte boundary), x = position + mis, so that a step, the positions of a
+// thread and every 16-byte vector start on a 16-byte boundary of global memory.
+struct SweepGeom {
+  const float* src;       // score of position 0
+  int e;                  // eligible positions [0, e)
+  int mis, n_chunks, pool, k;
+};
+
+__device__ __forceinline__ SweepGeom make_geom(const float* src, int e, int pool, int k) {
+  SweepGeom g;
+  g.src = src; g.e = e; g.pool = pool; g.k = k;
+  g.mis = (int)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u);
+  g.n_chunks = (e + g.mis + kChunk - 1) / kChunk;
+  return g;
+}
+
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// The 16 scores around this thread's 8 positions of step c: x in [xb - 4, xb + 12) with
+// xb = c*kChunk + 8*tid.  Positions outside [0, e) read as -infinity.
+__device__ __forceinline__ void load_window(const SweepGeom& g, int c, float4 (&w)[4]) {
+  const int p_first = c * kChunk + (int)threadIdx.x * kPerThread - 4 - g.mis;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int p0 = p_first + 4 * i;
+    if (p0 >= 0 && p0 + 3 < g.e) {
+      w[i] = __ldg(reinterpret_cast<const float4*>(g.src + p0));
     } else {
-      stage[i] = fill;
-    }
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-}
-
-// Pooled keys of this thread's kPerThread consecutive positions of the staged chunk.
-// stage[i] holds the score of position chunk_begin - h_lo + i (or the fill value).
-template <bool MAX7>
-__device__ __forceinline__ void chunk_keys(const float* stage, int pool, int k, uint32_t (&key)[kPerThread]) {
-  const int o = threadIdx.x * kPerThread;
-  if (MAX7) {
-    float w[16];
+      float t[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float4 v = *reinterpret_cast<const float4*>(stage + o + 4 * i);
-      w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
-    }
-#pragma unroll
-    for (int u = 0; u < kPerThread; ++u) {
-      const float a = fmaxf(fmaxf(w[u], w[u + 1]), fmaxf(w[u + 2], w[u + 3]));
-      const float b = fmaxf(fmaxf(w[u + 4], w[u + 5]), w[u + 6]);
-      key[u] = to_key(fmaxf(a, b));
-    }
-  } else {
-#pragma unroll
-    for (int u = 0; u < kPerThread; ++u) {
-      const float* wdw = stage + o + u;
-      float acc;
-      if (pool == SPEC_POOL_MAX) {
-        acc = wdw[0];
-        for (int t = 1; t < k; ++t) acc = fmaxf(acc, wdw[t]);
-      } else {
-        acc = 0.f;
-        for (int t = 0; t < k; ++t) acc += wdw[t];
-        acc = acc / (float)k;
-      }
-      key[u] = to_key(acc);
+      for (int q = 0; q < 4; ++q) t[q] = (p0 + q >= 0 && p0 + q < g.e) ? __ldg(g.src + p0 + q) : -INFINITY;
+      w[i] = make_float4(t[0], t[1], t[2], t[3]);
     }
   }
 }
 
-// Streams the pooled keys of the eligible range [0, e) chunk by chunk; f(key, j0) receives the
-// keys of positions j0 .. j0 + kPerThread - 1 (positions >= e carry no meaning).  f is called
-// by every thread the same number of times and may synchronise the CTA.
+// Max-pool of width 7 over the window: position u pools elements u + 1 .. u + 7.
+__device__ __forceinline__ void pool_max7(const float4 (&w4)[4], float (&val)[kPerThread]) {
+  static_assert(kPerThread == 8, "the window code is written for eight positions per thread");
+  const float w[16] = {w4[0].x, w4[0].y, w4[0].z, w4[0].w, w4[1].x, w4[1].y, w4[1].z, w4[1].w,
+                       w4[2].x, w4[2].y, w4[2].z, w4[2].w, w4[3].x, w4[3].y, w4[3].z, w4[3].w};
+  float t3[13];                                            // maxima of three neighbours, shared by the windows
+#pragma unroll
+  for (int i = 1; i < 13; ++i) t3[i] = fmax3(w[i], w[i + 1], w[i + 2]);
+#pragma unroll
+  for (int u = 0; u < kPerThread; ++u) val[u] = fmax3(t3[u + 1], t3[u + 4], w[u + 7]);
+}
+
+// Streams the pooled values of the eligible range step by step.  f(val, p0, edge, c) receives
+// the values of positions p0 .. p0 + kPerThread - 1 of step c; only when `edge` is set can
+// some of them lie outside [0, e) (they are then meaningless).  f is called by every thread
+// the same number of times and may synchronise the CTA.
 template <class F>
-__device__ __forceinline__ void sweep(const float* __restrict__ src, int e, int pool, int k, float* stages, F f) {
-  const int h_lo = k >> 1, span = kChunk + k - 1;
-  const float fill = pool == SPEC_POOL_MAX ? -INFINITY : 0.f;
-  const int n_chunks = (e + kChunk - 1) / kChunk;
-  const bool max7 = pool == SPEC_POOL_MAX && k == 7;
-  chunk_load(stages, src, e, 0, h_lo, span, fill);
-  for (int c = 0; c < n_chunks; ++c) {
-    float* stage = stages + (c & 1) * kStageFloats;
-    if (c + 1 < n_chunks) {
-      chunk_load(stages + ((c + 1) & 1) * kStageFloats, src, e, c + 1, h_lo, span, fill);
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
+__device__ __forceinline__ void sweep(const SweepGeom& g, F f) {
+  const bool max7 = g.pool == SPEC_POOL_MAX && g.k == 7;
+  float4 nxt[4];
+  if (max7) load_window(g, 0, nxt);
+  for (int c = 0; c < g.n_chunks; ++c) {
+    const int p0 = c * kChunk + (int)threadIdx.x * kPerThread - g.mis;
+    float val[kPerThread];
+    if (max7) {
+      float4 cur[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
+      if (c + 1 < g.n_chunks) load_window(g, c + 1, nxt);  // in flight while this step is processed
+      pool_max7(cur, val);
     } else {
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      // any other pooling: windows read element by element (L1 serves the overlap)
+#pragma unroll
+      for (int u = 0; u < kPerThread; ++u)
+        val[u] = (unsigned)(p0 + u) < (unsigned)g.e ? pooled_at(g.src, g.e, p0 + u, g.pool, g.k) : 0.f;
     }
-    __syncthreads();
-    uint32_t key[kPerThread];
-    if (max7) chunk_keys<true>(stage, pool, k, key); else chunk_keys<false>(stage, pool, k, key);
-    f(key, c * kChunk + (int)threadIdx.x * kPerThread);
-    __syncthreads();                                       // the stage may be refilled
+    const bool edge = (c == 0 && g.mis > 0) || c == g.n_chunks - 1;
+    f(val, p0, edge, c);
   }
 }
 
 // Finds the bin holding the need-th largest element of a histogram whose bins are spread
-// over the threads, bins_per_thread consecutive bins each (need >= 1, need <= total count).
-// Returns the bin and the number of elements in higher bins to every thread.
-__device__ __forceinline__ void locate_bin(const uint32_t* hist, int bins_per_thread, int need, int* wsum, int* out2,
+// over the threads, bins_per_thread consecutive bins each (need >= 1).  Returns the bin and
+// the number of elements in higher bins to every thread; false (outputs untouched) when the
+// histogram holds fewer than `need` elements.
+__device__ __forceinline__ bool locate_bin(const uint32_t* hist, int bins_per_thread, int need, int* wsum, int* out2,
                                            int& bin, int& above) {
   const int b0 = threadIdx.x * bins_per_thread;
+  __syncthreads();                                         // histogram complete, wsum free
+  if (threadIdx.x == 0) out2[0] = -1;
   int mine = 0;
   for (int i = 0; i < bins_per_thread; ++i) mine += (int)hist[b0 + i];
   int total;
@@ -332,9 +341,13 @@ __device__ __forceinline__ void locate_bin(const uint32_t* hist, int bins_per_th
     out2[1] = cum;
   }
   __syncthreads();
-  bin = out2[0];
-  above = out2[1];
+  const int found = out2[0];
+  const int cum = out2[1];
   __syncthreads();
+  if (found < 0) return false;
+  bin = found;
+  above = cum;
+  return true;
 }
 
 __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p) {
@@ -342,10 +355,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   uint32_t* top_hist = reinterpret_cast<uint32_t*>(smem_raw);            // sweep A; later the candidate keys
   uint32_t* cand_key = top_hist;
   int32_t* cand_idx = reinterpret_cast<int32_t*>(top_hist + kTopBins);
-  float* stages = reinterpret_cast<float*>(cand_idx + kCandCap);
-  int* wsum = reinterpret_cast<int*>(stages + 2 * kStageFloats);        // kSelWarps + 1 (+ 2 results)
-  int* out2 = wsum + kSelWarps + 1;
-  uint32_t* fin_hist = reinterpret_cast<uint32_t*>(stages);             // candidate passes, after the sweeps
+  uint32_t* fin_hist = reinterpret_cast<uint32_t*>(cand_idx + kCandCap); // candidate passes
+  int* wsum = reinterpret_cast<int*>(fin_hist + kFinBins);              // two buffers of kSelWarps, then two results
+  int* out2 = wsum + 2 * kSelWarps;
 
   const int unit = blockIdx.x;
   const int h = unit % p.H, l = (unit / p.H) % p.L, s = unit / (p.H * p.L);
@@ -359,51 +371,53 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   const float* src = p.scores + ((int64_t)l * p.H + h) * p.T + begin;
 
   if (take > 0 && take < e) {
+    const SweepGeom geom = make_geom(src, e, p.pool, p.pool_k);
     // ---- sweep A: which bin of the top kTopBits bits holds the take-th largest key
     int b1 = 0, above = 0;
     bool fits = true;
     if (e > kCandCap) {
       for (int i = tid; i < kTopBins; i += kSelThreads) top_hist[i] = 0;
       __syncthreads();
-      sweep(src, e, p.pool, p.pool_k, stages, [&](const uint32_t (&key)[kPerThread], int j0) {
-        uint32_t run_d = 0xffffffffu, run_c = 0;
+      // The take-th largest key of a prefix of the unit can only be below that of the whole
+      // unit, so the bin located on the chunks seen so far is a lower bound: keys under it
+      // are not counted any more (they would all hit the same few bins and serialise).
+      uint32_t floor_key = 0;
+      sweep(geom, [&](const float (&val)[kPerThread], int p0, bool edge, int c) {
+        // straight-line, predicated: once the floor is set only a few per cent of the keys count
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u) {
-          if (j0 + u < e) {
-            const uint32_t dg = key[u] >> (32 - kTopBits);
-            if (dg == run_d) {
-              ++run_c;
-            } else {
-              if (run_c) atomicAdd(&top_hist[run_d], run_c);
-              run_d = dg;
-              run_c = 1;
-            }
-          }
+          const uint32_t kk = to_key(val[u]);
+          if (kk >= floor_key && (!edge || (unsigned)(p0 + u) < (unsigned)e)) atomicAdd(&top_hist[kk >> (32 - kTopBits)], 1u);
         }
-        if (run_c) atomicAdd(&top_hist[run_d], run_c);
+        if (((c + 1) & c) == 0 || (c & 15) == 15) {        // after chunks 1, 2, 4, 8, 16, then every 16th
+          int fb, ab;
+          if (locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, fb, ab)) floor_key = (uint32_t)fb << (32 - kTopBits);
+        }
       });
-      locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, b1, above);
-      fits = above + (int)top_hist[b1] <= kCandCap;
+      fits = locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
+      fits = fits && above + (int)top_hist[b1] <= kCandCap;
       __syncthreads();                                     // top_hist is dead: its memory becomes cand_key
     }
     if (fits) {
       // ---- sweep B: candidates (keys in or above bin b1) in position order
       int n_cand = 0;
-      sweep(src, e, p.pool, p.pool_k, stages, [&](const uint32_t (&key)[kPerThread], int j0) {
-        int cnt = 0;
+      const uint32_t thr_key = (uint32_t)b1 << (32 - kTopBits);
+      sweep(geom, [&](const float (&val)[kPerThread], int p0, bool edge, int c) {
+        uint32_t take_mask = 0;
 #pragma unroll
-        for (int u = 0; u < kPerThread; ++u) cnt += (j0 + u < e) && (int)(key[u] >> (32 - kTopBits)) >= b1;
+        for (int u = 0; u < kPerThread; ++u)
+          if (to_key(val[u]) >= thr_key && (!edge || (unsigned)(p0 + u) < (unsigned)e)) take_mask |= 1u << u;
         int total;
-        int at = n_cand + block_exclusive_scan(cnt, wsum, total);
+        int at = n_cand + block_exclusive_scan(__popc(take_mask), wsum + (c & 1) * kSelWarps, total);
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u) {
-          if ((j0 + u < e) && (int)(key[u] >> (32 - kTopBits)) >= b1) {
-            cand_key[at] = key[u];
-            cand_idx[at] = j0 + u;
+          if ((take_mask & (1u << u)) && at < kCandCap) {
+            cand_key[at] = to_key(val[u]);
+            cand_idx[at] = p0 + u;
             ++at;
           }
         }
-        n_cand += total;
+        n_cand = min(n_cand + total, kCandCap);
       });
       // ---- remaining bits on the candidates only
       int known = e > kCandCap ? kTopBits : 0;
@@ -434,6 +448,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       int gt = 0, eq = 0;
       for (int i = i0; i < i1; ++i) { const uint32_t kk = cand_key[i]; gt += kk > T; eq += kk == T; }
       int total;
+      __syncthreads();
       const int packed = block_exclusive_scan(gt | (eq << 16), wsum, total);   // n_cand <= 8192 < 2^16
       int pre_gt = packed & 0xffff, pre_eq = packed >> 16;
       for (int i = i0; i < i1; ++i) {
@@ -449,7 +464,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     } else {
       // ---- too many keys share the leading bits: generic selection, keys recomputed per pass
       SelectScratch sc;
-      sc.hist = reinterpret_cast<uint32_t*>(stages);
+      sc.hist = top_hist;                                  // 16 KB + a few words of the 64 KB the candidates would use
       sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
       KeySource key;
       key.scores = src;
@@ -467,7 +482,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   if (p.count_out && tid == 0) p.count_out[unit] = take + forced;
 }
 
-constexpr int kTopkSmemBytes = kTopBins * 4 + kCandCap * 4 + 2 * kStageFloats * 4 + (kSelWarps + 1 + 2) * 4 + 16;
+constexpr int kTopkSmemBytes = kTopBins * 4 + kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2) * 4 + 16;
 
 // ---------------------------------------------------------------------- SpecPC ------
 
