@@ -190,22 +190,25 @@ struct TopkParams {
 
 // ------------------------------------------------------ streaming pool + top-C ------
 //
-// One CTA per (sequence, layer, KV head) unit, any length.  The unit's scores are streamed
-// twice, kChunk positions per step, straight from global memory into registers (16-byte
-// loads, the next step's loads in flight while the current one is processed):
-//   sweep A  pooled keys -> histogram of their top kTopBits bits (shared-memory atomics);
-//            the bin holding the C-th largest key is located;
-//   sweep B  (served by L2) every key in or above that bin is appended, in position order,
-//            to a candidate list in shared memory;
-// the remaining bits are then resolved by radix passes over the candidates only, and the
-// winners are written in ascending position.  Units with at most kCandCap positions skip
-// sweep A.  If the candidates do not fit (many nearly equal scores), the unit falls back to
-// the generic multi-pass selection that recomputes keys from global memory.
-constexpr int kChunk = 4096;                      // positions per step: 8 consecutive per thread
-constexpr int kPerThread = kChunk / kSelThreads;
+// One CTA per (sequence, layer, KV head) unit, any length.  The unit's scores are read once.
+// Every warp owns a contiguous range of positions and streams it on its own, kWarpStep
+// positions per step, straight from global memory into registers (16-byte loads, the next
+// step's loads in flight while the current one is processed), with no CTA-wide barrier per
+// step.  Every pooled key at or above a rising floor is counted in a shared histogram of the
+// keys' top kTopBits bits and appended, in position order, to the warp's candidate list in
+// shared memory; the floor is the bin that holds the C-th largest key of the positions seen so
+// far and is raised at a few CTA-wide synchronisation points.  After the sweep the remaining
+// bits are resolved by radix passes over the candidates only, and the winners are written in
+// ascending position (warp lists are in position order and so is their concatenation).  If
+// the candidates do not fit (many nearly equal scores, or c_max beyond a few thousand), the
+// unit falls back to the generic multi-pass selection that recomputes keys from global memory.
+constexpr int kPerThread = 8;                     // consecutive positions per thread and step
+constexpr int kWarpStep = 32 * kPerThread;        // positions per warp and step
 constexpr int kTopBits = 13;
 constexpr int kTopBins = 1 << kTopBits;
-constexpr int kCandCap = 8192;
+constexpr int kTopHistWords = kTopBins + (kTopBins >> 8) * 4;   // four words of padding per 256 bins
+constexpr int kCandCap = 7168;
+constexpr int kWarpCap = kCandCap / kSelWarps;    // candidate entries per warp
 constexpr int kFinBins = 1024;                    // histogram of the candidate passes (10 bits)
 
 // Block-wide exclusive scan of one int per thread; total returned to every thread.
@@ -234,20 +237,23 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int& total
   return before + incl - v;
 }
 
-// Geometry of the sweeps.  Positions are shifted by the unit's misalignment `mis` (0..3
-// elements from a 16-byte boundary), x = position + mis, so that a step, the positions of a
-// thread and every 16-byte vector start on a 16-byte boundary of global memory.
+// Geometry of the sweep.  Positions are shifted by the unit's misalignment `mis` (0..3
+// elements from a 16-byte boundary), x = position + mis, so that the positions of a thread and
+// every 16-byte vector start on a 16-byte boundary of global memory.  Warp w streams
+// x in [w * span, (w + 1) * span), span a multiple of kWarpStep.
 struct SweepGeom {
   const float* src;       // score of position 0
   int e;                  // eligible positions [0, e)
-  int mis, n_chunks, pool, k;
+  int mis, span, n_steps, pool, k;
 };
 
 __device__ __forceinline__ SweepGeom make_geom(const float* src, int e, int pool, int k) {
   SweepGeom g;
   g.src = src; g.e = e; g.pool = pool; g.k = k;
   g.mis = (int)((reinterpret_cast<uintptr_t>(src) >> 2) & 3u);
-  g.n_chunks = (e + g.mis + kChunk - 1) / kChunk;
+  const int per_warp = (e + g.mis + kSelWarps - 1) / kSelWarps;
+  g.n_steps = (per_warp + kWarpStep - 1) / kWarpStep;
+  g.span = g.n_steps * kWarpStep;
   return g;
 }
 
@@ -257,19 +263,23 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
-// The 16 scores around this thread's 8 positions of step c: x in [xb - 4, xb + 12) with
-// xb = c*kChunk + 8*tid.  Positions outside [0, e) read as -infinity.
-__device__ __forceinline__ void load_window(const SweepGeom& g, int c, float4 (&w)[4]) {
-  const int p_first = c * kChunk + (int)threadIdx.x * kPerThread - 4 - g.mis;
+// The 16 scores around the 8 positions that start at x = xb: x in [xb - 4, xb + 12).
+// Positions outside [0, e) read as -infinity.
+__device__ __forceinline__ void load_window(const SweepGeom& g, int xb, float4 (&w)[4]) {
+  const int p_first = xb - 4 - g.mis;
+  if (p_first >= 0 && p_first + 15 < g.e) {
+    const float4* v = reinterpret_cast<const float4*>(g.src + p_first);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int p0 = p_first + 4 * i;
-    if (p0 >= 0 && p0 + 3 < g.e) {
-      w[i] = __ldg(reinterpret_cast<const float4*>(g.src + p0));
-    } else {
+    for (int i = 0; i < 4; ++i) w[i] = __ldg(v + i);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
       float t[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) t[q] = (p0 + q >= 0 && p0 + q < g.e) ? __ldg(g.src + p0 + q) : -INFINITY;
+      for (int q = 0; q < 4; ++q) {
+        const int pp = p_first + 4 * i + q;
+        t[q] = (pp >= 0 && pp < g.e) ? __ldg(g.src + pp) : -INFINITY;
+      }
       w[i] = make_float4(t[0], t[1], t[2], t[3]);
     }
   }
@@ -287,53 +297,28 @@ __device__ __forceinline__ void pool_max7(const float4 (&w4)[4], float (&val)[kP
   for (int u = 0; u < kPerThread; ++u) val[u] = fmax3(t3[u + 1], t3[u + 4], w[u + 7]);
 }
 
-// Streams the pooled values of the eligible range step by step.  f(val, p0, edge, c) receives
-// the values of positions p0 .. p0 + kPerThread - 1 of step c; only when `edge` is set can
-// some of them lie outside [0, e) (they are then meaningless).  f is called by every thread
-// the same number of times and may synchronise the CTA.
-template <class F>
-__device__ __forceinline__ void sweep(const SweepGeom& g, F f) {
-  const bool max7 = g.pool == SPEC_POOL_MAX && g.k == 7;
-  float4 nxt[4];
-  if (max7) load_window(g, 0, nxt);
-  for (int c = 0; c < g.n_chunks; ++c) {
-    const int p0 = c * kChunk + (int)threadIdx.x * kPerThread - g.mis;
-    float val[kPerThread];
-    if (max7) {
-      float4 cur[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
-      if (c + 1 < g.n_chunks) load_window(g, c + 1, nxt);  // in flight while this step is processed
-      pool_max7(cur, val);
-    } else {
-      // any other pooling: windows read element by element (L1 serves the overlap)
-#pragma unroll
-      for (int u = 0; u < kPerThread; ++u)
-        val[u] = (unsigned)(p0 + u) < (unsigned)g.e ? pooled_at(g.src, g.e, p0 + u, g.pool, g.k) : 0.f;
-    }
-    const bool edge = (c == 0 && g.mis > 0) || c == g.n_chunks - 1;
-    f(val, p0, edge, c);
-  }
-}
+// Word of bin b in the top-bits histogram: every lane of a warp scans 256 consecutive bins
+// with 16-byte loads, and the padding staggers the lanes over the memory banks.
+__device__ __forceinline__ int top_word(uint32_t b) { return (int)(b + ((b >> 8) << 2)); }
 
 // Finds the bin holding the need-th largest element of a histogram whose bins are spread
-// over the threads, bins_per_thread consecutive bins each (need >= 1).  Returns the bin and
+// over the threads, bins_per_thread consecutive bins each starting at my_bins (need >= 1).  Returns the bin and
 // the number of elements in higher bins to every thread; false (outputs untouched) when the
 // histogram holds fewer than `need` elements.
-__device__ __forceinline__ bool locate_bin(const uint32_t* hist, int bins_per_thread, int need, int* wsum, int* out2,
+__device__ __forceinline__ bool locate_bin(const uint32_t* my_bins, int bins_per_thread, int need, int* wsum, int* out2,
                                            int& bin, int& above) {
   const int b0 = threadIdx.x * bins_per_thread;
   __syncthreads();                                         // histogram complete, wsum free
   if (threadIdx.x == 0) out2[0] = -1;
   int mine = 0;
-  for (int i = 0; i < bins_per_thread; ++i) mine += (int)hist[b0 + i];
+  for (int i = 0; i < bins_per_thread; ++i) mine += (int)my_bins[i];
   int total;
   const int below = block_exclusive_scan(mine, wsum, total);
   const int over = total - below - mine;                   // elements in bins above my range
   if (over < need && need <= over + mine) {
     int cum = over, b = bins_per_thread - 1;
     for (; b > 0; --b) {
-      const int hcount = (int)hist[b0 + b];
+      const int hcount = (int)my_bins[b];
       if (cum + hcount >= need) break;
       cum += hcount;
     }
@@ -350,14 +335,22 @@ __device__ __forceinline__ bool locate_bin(const uint32_t* hist, int bins_per_th
   return true;
 }
 
+// Shared memory: top histogram, candidate keys and positions, candidate-pass histogram, a few
+// words of bookkeeping, then the parked groups (values and first positions) of all warps.
+constexpr int kTopkPendOffset = (kTopHistWords * 4 + 2 * kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2 + 1) * 4 + 15) / 16 * 16;
+constexpr int kTopkSmemBytes = kTopkPendOffset + kSelWarps * 32 * (kPerThread + 1) * 4;
+
 __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  uint32_t* top_hist = reinterpret_cast<uint32_t*>(smem_raw);            // sweep A; later the candidate keys
-  uint32_t* cand_key = top_hist;
-  int32_t* cand_idx = reinterpret_cast<int32_t*>(top_hist + kTopBins);
+  uint32_t* top_hist = reinterpret_cast<uint32_t*>(smem_raw);            // histogram of the keys' top bits
+  uint32_t* cand_key = top_hist + kTopHistWords;                        // [kSelWarps][kWarpCap]
+  int32_t* cand_idx = reinterpret_cast<int32_t*>(cand_key + kCandCap);
   uint32_t* fin_hist = reinterpret_cast<uint32_t*>(cand_idx + kCandCap); // candidate passes
-  int* wsum = reinterpret_cast<int*>(fin_hist + kFinBins);              // two buffers of kSelWarps, then two results
-  int* out2 = wsum + 2 * kSelWarps;
+  int* wsum = reinterpret_cast<int*>(fin_hist + kFinBins);              // kSelWarps, then two results, then flags
+  int* out2 = wsum + kSelWarps;
+  int* wcnt = out2 + 2;                                                  // [kSelWarps] list lengths, then the overflow flag
+  int* overflow = wcnt + kSelWarps;
+  float* pend = reinterpret_cast<float*>(smem_raw + kTopkPendOffset);    // parked groups of all warps
 
   const int unit = blockIdx.x;
   const int h = unit % p.H, l = (unit / p.H) % p.L, s = unit / (p.H * p.L);
@@ -367,74 +360,206 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   const int e = n - forced;
   const int take = min(p.c_max - forced, e);
   int32_t* idx = p.idx_out + (int64_t)unit * p.c_max;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t lt_mask = (1u << lane) - 1u;
   const float* src = p.scores + ((int64_t)l * p.H + h) * p.T + begin;
 
   if (take > 0 && take < e) {
-    const SweepGeom geom = make_geom(src, e, p.pool, p.pool_k);
-    // ---- sweep A: which bin of the top kTopBits bits holds the take-th largest key
-    int b1 = 0, above = 0;
-    bool fits = true;
-    if (e > kCandCap) {
-      for (int i = tid; i < kTopBins; i += kSelThreads) top_hist[i] = 0;
-      __syncthreads();
-      // The take-th largest key of a prefix of the unit can only be below that of the whole
-      // unit, so the bin located on the chunks seen so far is a lower bound: keys under it
-      // are not counted any more (they would all hit the same few bins and serialise).
-      uint32_t floor_key = 0;
-      sweep(geom, [&](const float (&val)[kPerThread], int p0, bool edge, int c) {
-        // straight-line, predicated: once the floor is set only a few per cent of the keys count
+    const SweepGeom g = make_geom(src, e, p.pool, p.pool_k);
+    for (int i = tid; i < kTopHistWords; i += kSelThreads) top_hist[i] = 0;
+    if (tid == 0) *overflow = 0;
+    __syncthreads();
+    uint32_t* ck = cand_key + warp * kWarpCap;
+    int32_t* ci = cand_idx + warp * kWarpCap;
+    const bool max7 = g.pool == SPEC_POOL_MAX && g.k == 7;
+    // ---- the sweep.  The take-th largest key of the positions seen so far can only be below
+    // that of the whole unit, so the bin that holds it is a floor: keys under it are out.
+    uint32_t floor_key = 0;
+    int cnt = 0;                                             // entries in my warp's list (warp-uniform)
+    const int x_warp = warp * g.span + lane * kPerThread;
+
+    // One step of my warp: the pooled values of positions p0 .. p0 + 7 of every lane.
+    // Raises my warp's floor to the bin that holds the take-th largest of the keys counted so
+    // far, read from the shared histogram without stopping the other warps.  Their updates can
+    // only add keys, so the bin found is still a lower bound.
+    auto warp_refloor = [&]() {
+      constexpr int kBinsPerLane = kTopBins / 32;
+      static_assert(kBinsPerLane == 256, "the padding of the histogram assumes 256 bins per lane");
+      const uint32_t* hb = top_hist + lane * (kBinsPerLane + 4);
+      int mine = 0;
+      for (int i = 0; i < kBinsPerLane; i += 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(hb + i);
+        mine += (int)(v.x + v.y + v.z + v.w);
+      }
+      int suffix = mine;                                     // keys in my bins and in those of higher lanes
 #pragma unroll
-        for (int u = 0; u < kPerThread; ++u) {
-          const uint32_t kk = to_key(val[u]);
-          if (kk >= floor_key && (!edge || (unsigned)(p0 + u) < (unsigned)e)) atomicAdd(&top_hist[kk >> (32 - kTopBits)], 1u);
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_down_sync(0xffffffffu, suffix, o);
+        if (lane + o < 32) suffix += t;
+      }
+      const bool here = suffix - mine < take && take <= suffix;
+      int bin = -1;
+      if (here) {
+        int cum = suffix - mine;
+        bin = kBinsPerLane - 1;
+        for (; bin > 0; --bin) {
+          cum += (int)hb[bin];
+          if (cum >= take) break;
         }
-        if (((c + 1) & c) == 0 || (c & 15) == 15) {        // after chunks 1, 2, 4, 8, 16, then every 16th
-          int fb, ab;
-          if (locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, fb, ab)) floor_key = (uint32_t)fb << (32 - kTopBits);
-        }
-      });
-      fits = locate_bin(top_hist, kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
-      fits = fits && above + (int)top_hist[b1] <= kCandCap;
-      __syncthreads();                                     // top_hist is dead: its memory becomes cand_key
-    }
-    if (fits) {
-      // ---- sweep B: candidates (keys in or above bin b1) in position order
-      int n_cand = 0;
-      const uint32_t thr_key = (uint32_t)b1 << (32 - kTopBits);
-      sweep(geom, [&](const float (&val)[kPerThread], int p0, bool edge, int c) {
-        uint32_t take_mask = 0;
+        bin += lane * kBinsPerLane;
+      }
+      const uint32_t who = __ballot_sync(0xffffffffu, here);
+      if (who) {
+        const uint32_t fk = (uint32_t)__shfl_sync(0xffffffffu, bin, __ffs(who) - 1) << (32 - kTopBits);
+        if (fk > floor_key) floor_key = fk;
+      }
+    };
+
+    // Ordered in-place filter of my warp's list against the current floor.
+    auto filter_list = [&]() {
+      int kept = 0;
+      for (int r = 0; r < cnt; r += 32) {
+        const int i = r + lane;
+        const uint32_t kk = i < cnt ? ck[i] : 0u;
+        const int32_t ix = i < cnt ? ci[i] : 0;
+        const bool keep = i < cnt && kk >= floor_key;
+        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+        __syncwarp();                                      // every lane holds its entry before any is overwritten
+        if (keep) { const int w = kept + __popc(bal & lt_mask); ck[w] = kk; ci[w] = ix; }
+        kept += __popc(bal);
+        __syncwarp();
+      }
+      cnt = kept;
+    };
+
+    // Groups (the eight pooled values of one lane and one step) that hold at least one key at
+    // or above the floor are parked in a small per-warp buffer and dealt with 32 at a time,
+    // one group per lane, so that the per-key work runs with full warps instead of once per
+    // step for a handful of keys.
+    float* pend_val = pend + warp * (32 * kPerThread);      // [32 groups][8 values]
+    int* pend_p0 = reinterpret_cast<int*>(pend + kSelWarps * 32 * kPerThread) + warp * 32;
+    int n_pend = 0;                                          // parked groups (warp-uniform)
+
+    auto expand = [&]() {
+      if (n_pend == 0) return;
+      const bool have = lane < n_pend;
+      float val[kPerThread];
+      const float4 v0 = *reinterpret_cast<const float4*>(pend_val + lane * kPerThread);
+      const float4 v1 = *reinterpret_cast<const float4*>(pend_val + lane * kPerThread + 4);
+      val[0] = v0.x; val[1] = v0.y; val[2] = v0.z; val[3] = v0.w;
+      val[4] = v1.x; val[5] = v1.y; val[6] = v1.z; val[7] = v1.w;
+      const int p0 = pend_p0[lane];
+      uint32_t take_mask = 0;
+      if (have) {
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u)
-          if (to_key(val[u]) >= thr_key && (!edge || (unsigned)(p0 + u) < (unsigned)e)) take_mask |= 1u << u;
-        int total;
-        int at = n_cand + block_exclusive_scan(__popc(take_mask), wsum + (c & 1) * kSelWarps, total);
+          if (to_key(val[u]) >= floor_key && (unsigned)(p0 + u) < (unsigned)e) take_mask |= 1u << u;
+      }
+      const int mine = __popc(take_mask);
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+      for (int u = 0; u < kPerThread; ++u)
+        if (take_mask & (1u << u)) atomicAdd(&top_hist[top_word(to_key(val[u]) >> (32 - kTopBits))], 1u);
+      if (cnt + total > kWarpCap) filter_list();
+      if (cnt + total > kWarpCap) { warp_refloor(); filter_list(); }   // my list alone is too long: fresher floor
+      if (cnt + total <= kWarpCap) {
+        int at = cnt + incl - mine;
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u) {
-          if ((take_mask & (1u << u)) && at < kCandCap) {
-            cand_key[at] = to_key(val[u]);
-            cand_idx[at] = p0 + u;
+          if (take_mask & (1u << u)) {
+            ck[at] = to_key(val[u]);
+            ci[at] = p0 + u;
             ++at;
           }
         }
-        n_cand = min(n_cand + total, kCandCap);
-      });
-      // ---- remaining bits on the candidates only
-      int known = e > kCandCap ? kTopBits : 0;
-      uint32_t prefix = e > kCandCap ? (uint32_t)b1 << (32 - kTopBits) : 0u;
-      uint32_t mask = e > kCandCap ? ~((1u << (32 - kTopBits)) - 1u) : 0u;
+        cnt += total;
+      } else if (lane == 0) {
+        *overflow = 1;                                       // the list is lost: the unit takes the generic path
+      }
+      n_pend = 0;
+      __syncwarp();
+    };
+
+    // One step of my warp: the pooled values of positions p0 .. p0 + 7 of every lane.
+    auto process = [&](const float (&val)[kPerThread], int p0, int st) {
+      const float vmax = fmax3(fmax3(val[0], val[1], val[2]), fmax3(val[3], val[4], val[5]), fmaxf(val[6], val[7]));
+      const bool hot = p0 + kPerThread > 0 && p0 < e && to_key(vmax) >= floor_key;
+      const uint32_t hot_lanes = __ballot_sync(0xffffffffu, hot);
+      if (hot_lanes) {
+        const int n_hot = __popc(hot_lanes);
+        if (n_pend + n_hot > 32) expand();
+        if (hot) {
+          const int slot = n_pend + __popc(hot_lanes & lt_mask);
+          *reinterpret_cast<float4*>(pend_val + slot * kPerThread) = make_float4(val[0], val[1], val[2], val[3]);
+          *reinterpret_cast<float4*>(pend_val + slot * kPerThread + 4) = make_float4(val[4], val[5], val[6], val[7]);
+          pend_p0[slot] = p0;
+        }
+        n_pend += n_hot;
+        __syncwarp();
+      }
+      if (((st + 1) & st) == 0 || (st & 31) == 31) expand();  // the histogram must be complete for the floor
+      if (((st + 1) & st) == 0 || (st & 31) == 31) {       // after steps 0, 1, 3, 7, 15, 31, then every 32nd
+        int fb, ab;
+        if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, fb, ab))
+          floor_key = max(floor_key, (uint32_t)fb << (32 - kTopBits));
+      }
+    };
+
+    if (max7) {
+      // two steps of loads in flight per thread; a window's registers are refilled as soon as
+      // it has been pooled
+      float4 wa[4], wb[4];
+      load_window(g, x_warp, wa);
+      if (g.n_steps > 1) load_window(g, x_warp + kWarpStep, wb);
+      for (int st = 0; st < g.n_steps; st += 2) {
+        float val[kPerThread];
+        pool_max7(wa, val);
+        if (st + 2 < g.n_steps) load_window(g, x_warp + (st + 2) * kWarpStep, wa);
+        process(val, x_warp + st * kWarpStep - g.mis, st);
+        if (st + 1 < g.n_steps) {
+          pool_max7(wb, val);
+          if (st + 3 < g.n_steps) load_window(g, x_warp + (st + 3) * kWarpStep, wb);
+          process(val, x_warp + (st + 1) * kWarpStep - g.mis, st + 1);
+        }
+      }
+    } else {
+      // any other pooling: windows read element by element (L1 serves the overlap)
+      for (int st = 0; st < g.n_steps; ++st) {
+        const int p0 = x_warp + st * kWarpStep - g.mis;
+        float val[kPerThread];
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u)
+          val[u] = (unsigned)(p0 + u) < (unsigned)e ? pooled_at(src, e, p0 + u, g.pool, g.k) : 0.f;
+        process(val, p0, st);
+      }
+    }
+    expand();
+    if (lane == 0) wcnt[warp] = cnt;
+    int b1 = 0, above = 0;
+    bool fits = locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
+    fits = fits && *overflow == 0;
+    if (fits) {
+      // ---- remaining bits on the candidates only (every warp walks its own list)
+      int known = kTopBits;
+      uint32_t prefix = (uint32_t)b1 << (32 - kTopBits);
+      uint32_t mask = ~((1u << (32 - kTopBits)) - 1u);
       int remaining = take - above;
       while (known < 32) {
         const int w = min(10, 32 - known), shift = 32 - known - w;
         for (int i = tid; i < kFinBins; i += kSelThreads) fin_hist[i] = 0;
         __syncthreads();
-        for (int i = tid; i < n_cand; i += kSelThreads) {
-          const uint32_t kk = cand_key[i];
+        for (int i = lane; i < cnt; i += 32) {
+          const uint32_t kk = ck[i];
           if ((kk & mask) == prefix) atomicAdd(&fin_hist[(kk >> shift) & ((1u << w) - 1u)], 1u);
         }
-        __syncthreads();
         int dg, ab;
-        locate_bin(fin_hist, kFinBins / kSelThreads, remaining, wsum, out2, dg, ab);
+        locate_bin(fin_hist + tid * (kFinBins / kSelThreads), kFinBins / kSelThreads, remaining, wsum, out2, dg, ab);
         remaining -= ab;
         prefix |= (uint32_t)dg << shift;
         mask |= ((1u << w) - 1u) << shift;
@@ -443,28 +568,34 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       // ---- ordered emission: key > T, or key == T among the first `remaining` equal keys
       const uint32_t T = prefix;
       const int need_eq = remaining;
-      const int per = (n_cand + kSelThreads - 1) / kSelThreads;
-      const int i0 = min(tid * per, n_cand), i1 = min(i0 + per, n_cand);
       int gt = 0, eq = 0;
-      for (int i = i0; i < i1; ++i) { const uint32_t kk = cand_key[i]; gt += kk > T; eq += kk == T; }
-      int total;
+      for (int i = lane; i < cnt; i += 32) { const uint32_t kk = ck[i]; gt += kk > T; eq += kk == T; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        gt += __shfl_xor_sync(0xffffffffu, gt, o);
+        eq += __shfl_xor_sync(0xffffffffu, eq, o);
+      }
+      __syncthreads();                                     // wcnt no longer needed: reuse it for (gt, eq) per warp
+      if (lane == 0) wcnt[warp] = gt | (eq << 16);         // a list holds at most kWarpCap < 2^16 entries
       __syncthreads();
-      const int packed = block_exclusive_scan(gt | (eq << 16), wsum, total);   // n_cand <= 8192 < 2^16
-      int pre_gt = packed & 0xffff, pre_eq = packed >> 16;
-      for (int i = i0; i < i1; ++i) {
-        const uint32_t kk = cand_key[i];
-        if (kk > T) {
-          idx[pre_gt + min(pre_eq, need_eq)] = cand_idx[i];
-          ++pre_gt;
-        } else if (kk == T) {
-          if (pre_eq < need_eq) idx[pre_gt + pre_eq] = cand_idx[i];
-          ++pre_eq;
-        }
+      int pre_gt = 0, pre_eq = 0;
+      for (int w = 0; w < warp; ++w) { const int x = wcnt[w]; pre_gt += x & 0xffff; pre_eq += x >> 16; }
+      for (int r = 0; r < cnt; r += 32) {
+        const int i = r + lane;
+        const uint32_t kk = i < cnt ? ck[i] : 0u;
+        const bool is_gt = i < cnt && kk > T, is_eq = i < cnt && kk == T;
+        const uint32_t bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
+        const int my_gt = pre_gt + __popc(bg & lt_mask), my_eq = pre_eq + __popc(be & lt_mask);
+        if (is_gt) idx[my_gt + min(my_eq, need_eq)] = ci[i];
+        else if (is_eq && my_eq < need_eq) idx[my_gt + my_eq] = ci[i];
+        pre_gt += __popc(bg);
+        pre_eq += __popc(be);
       }
     } else {
-      // ---- too many keys share the leading bits: generic selection, keys recomputed per pass
+      // ---- candidates lost or too many keys share the leading bits: generic selection
+      __syncthreads();
       SelectScratch sc;
-      sc.hist = top_hist;                                  // 16 KB + a few words of the 64 KB the candidates would use
+      sc.hist = cand_key;                                  // 16 KB + a few words of the 64 KB of the candidate lists
       sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
       KeySource key;
       key.scores = src;
@@ -482,7 +613,6 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   if (p.count_out && tid == 0) p.count_out[unit] = take + forced;
 }
 
-constexpr int kTopkSmemBytes = kTopBins * 4 + kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2) * 4 + 16;
 
 // ---------------------------------------------------------------------- SpecPC ------
 

@@ -179,6 +179,24 @@ def test_topk_streaming_regime_long_sequence(B, W, oracle):
     run_topk_case(B, W, oracle, scores, [0, 70001], 0, 7, 2048, 32)
 
 
+def test_topk_clustered_keys_large_budget_and_odd_offsets(B, W, oracle):
+    rng = np.random.default_rng(7)
+    # every heavy key inside the range one warp streams: its candidate list overflows and is re-filtered
+    scores = (rng.random((1, 2, 100000)).astype(np.float32) * 0.01)
+    scores[:, :, 1000:4000] += rng.random((1, 2, 3000)).astype(np.float32) + 1.0
+    run_topk_case(B, W, oracle, scores, [0, 100000], 0, 7, 2048, 0)
+    # ascending scores: every new position is a new maximum
+    ramp = np.linspace(0.0, 1.0, 60000, dtype=np.float32)[None, None, :].repeat(2, axis=1)
+    run_topk_case(B, W, oracle, ramp, [0, 60000], 0, 7, 1024, 0)
+    # a budget beyond the candidate lists: generic selection
+    scores = rng.random((1, 2, 50000)).astype(np.float32) ** 3
+    run_topk_case(B, W, oracle, scores, [0, 50000], 0, 7, 6000, 0)
+    # sequence starts that are not multiples of four elements (16-byte loads need realignment)
+    scores = rng.random((2, 2, 4099 + 33333 + 12345)).astype(np.float32) ** 5
+    run_topk_case(B, W, oracle, scores, [0, 4099, 4099 + 33333, 4099 + 33333 + 12345], 0, 7, 512, 0)
+    run_topk_case(B, W, oracle, scores, [0, 4099, 4099 + 33333, 4099 + 33333 + 12345], 0, 7, 512, 40)
+
+
 def test_topk_avg_pool_within_band(B, W, oracle):
     rng = np.random.default_rng(3)
     scores = rng.random((1, 2, 3000)).astype(np.float32) ** 4
