@@ -32,6 +32,32 @@ METRIC = "prompt_tokens_scored_and_compacted_per_s_all_layers"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per layer of the workload, from the ncu
+# captures summarised under profiles/ (small cases; traffic grows in proportion to the layers), with the
+# first 16 hex digits of the SHA-256 of the kernel source the capture was taken on.  A changed source
+# makes the figure stale and it is reported as null.
+NCU_TRAFFIC = {
+    # workload index -> {kernel group: (bytes per layer, source file, source hash)}
+    1: {"score": ((138.74e6 + 7.86e6 + 140.83e6 + 3.89e6) / 4, "score.cu", "77e44f053bbad4ca")},
+    2: {"select": (33.71e6 / 8, "select.cu", "7fc357d2b50fe8ef"),
+        "gather": ((67.65e6 + 17.14e6) / 8, "compact.cu", "cfd00eb467119c19")},
+}
+
+
+def ncu_traffic(config: int, group: str, n_layers: int):
+    import hashlib
+    ent = NCU_TRAFFIC.get(config, {}).get(group)
+    if ent is None:
+        return None
+    per_layer, src, digest = ent
+    try:
+        with open(os.path.join(ROOT, "paper_2506_08373_b200", "csrc", src), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != digest:
+                return None
+    except OSError:
+        return None
+    return per_layer * n_layers
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -326,14 +352,17 @@ def main(argv=None):
     roofline = {"bound": "tensor", "kernel": "spec_score: score_kernel<1> + merge + score_kernel<2>",
                 "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
                 "peak_source": peak_src + " (burst cuBLAS bf16)", "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
-                "achieved_one_contraction": tf / 2, "ms": t_score, "traffic": None}
+                "achieved_one_contraction": tf / 2, "ms": t_score,
+                "algorithmic_bytes": work["score_hbm_bytes"], "traffic": ncu_traffic(args.config, "score", st.L)}
     hbm_bytes = work["select_bytes"] + work["gather_bytes"]
     gbs = hbm_bytes / ((t_select + t_gather) * 1e-3) / 1e9
     roofline_hbm = {"bound": "hbm", "kernel": "pool_topk_kernel + compact_kernel" if not st.specpc else "token_reduce + specpc_keep",
                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": peak_src + " (copy)", "ms_select": t_select, "ms_gather": t_gather,
                     "gather_gbs": (work["gather_bytes"] / (t_gather * 1e-3) / 1e9) if t_gather > 0 and work["gather_bytes"] else None,
-                    "traffic": None}
+                    "algorithmic_bytes": hbm_bytes,
+                    "traffic": (None if st.specpc or ncu_traffic(args.config, "select", st.L) is None or ncu_traffic(args.config, "gather", st.L) is None
+                                else ncu_traffic(args.config, "select", st.L) + ncu_traffic(args.config, "gather", st.L))}
 
     line = {"metric": METRIC, "value": job_value(tokens, K, world, total_ms), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
