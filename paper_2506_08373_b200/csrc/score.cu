@@ -39,11 +39,21 @@ constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_POLY_PAIRS
 #define SPEC_POLY_PAIRS 3
 #endif
+#ifndef SPEC_POLY_SCALAR
+#define SPEC_POLY_SCALAR 0
+#endif
+#ifndef SPEC_SCALAR_ACC
+#define SPEC_SCALAR_ACC 0
+#endif
 #ifndef SPEC_LOAD_AHEAD
 #define SPEC_LOAD_AHEAD 0
 #endif
 constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes
-constexpr bool kLoadAhead = SPEC_LOAD_AHEAD;  // fetch a work item's second 32 columns before the math on the first
+#ifndef SPEC_LOAD_AHEAD2
+#define SPEC_LOAD_AHEAD2 0
+#endif
+constexpr bool kLoadAhead = SPEC_LOAD_AHEAD;    // pass 1: fetch a work item's second 32 columns before the math on the first
+constexpr bool kLoadAhead2 = SPEC_LOAD_AHEAD2;  // pass 2: the same
 constexpr int kBufCols = 128;
 constexpr int kNumBufs = 4;
 constexpr int kTileKeys = 128;
@@ -92,20 +102,32 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait.  Returns false when another role has given up or the time limit passed.  The
 // suspend-time hint lets the hardware park the thread until the phase completes instead of
 // spinning in the issue slots the epilogue warps need.
-__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const uint32_t addr = smem_u32(bar);
   unsigned long long t0 = 0;
-  for (;;) {
+  for (uint32_t it = 1;; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
         : "=r"(ok) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
     if (ok) return true;
-    if (*abort_flag) return false;
-    const unsigned long long now = global_ns();
-    if (t0 == 0) t0 = now;
-    else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    if ((it & 7u) == 0) {                                   // every failed wait already lasted up to the hint
+      if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
   }
+}
+
+// The common case, a phase that has already completed, costs one non-blocking test inline.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  if (ok) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -250,6 +272,20 @@ __device__ __forceinline__ float2 ex2_mufu2(float2 x) { return make_float2(ex2(x
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic with relative error 7.5e-5,
 // then n is added into the exponent field.  x is clamped at -125 so the exponent cannot wrap.
 __device__ __forceinline__ float2 ex2_poly2(float2 x) {
+#if SPEC_POLY_SCALAR
+  // range reduction packed, polynomial per lane: scalar FFMA takes its coefficients as immediates,
+  // the packed form needs every constant pair in registers
+  x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
+  const float2 big = splat2(12582912.f), minus1 = splat2(-1.f);
+  const float2 xr = __fadd2_rn(x, big);
+  const float2 n = __ffma2_rn(big, minus1, xr);
+  const float2 f = __ffma2_rn(n, minus1, x);
+  float q0 = fmaf(f.x, 0.0551713221f, 0.2426105440f), q1 = fmaf(f.y, 0.0551713221f, 0.2426105440f);
+  q0 = fmaf(q0, f.x, 0.6932609677f); q1 = fmaf(q1, f.y, 0.6932609677f);
+  q0 = fmaf(q0, f.x, 0.9999281168f); q1 = fmaf(q1, f.y, 0.9999281168f);
+  return make_float2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(xr.x) << 23)),
+                     __uint_as_float(__float_as_uint(q1) + (__float_as_uint(xr.y) << 23)));
+#else
   x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
   const float2 xr = __fadd2_rn(x, splat2(12582912.f));
   const float2 n = __fadd2_rn(xr, splat2(-12582912.f));
@@ -259,6 +295,7 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
   q = __ffma2_rn(q, f, splat2(0.9999281168f));
   return make_float2(__uint_as_float(__float_as_uint(q.x) + (__float_as_uint(xr.x) << 23)),
                      __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(xr.y) << 23)));
+#endif
 }
 // Pair i (0..15) of a 32-element block: kPolyPairs of them, evenly spread, avoid the MUFU unit.
 __device__ __forceinline__ constexpr bool poly_pair(int i) {
@@ -286,6 +323,16 @@ __device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid,
   z *= ex2(m - mn);                                        // first block: 0 * 2^-inf = 0
   m = mn;
   const float2 a2 = splat2(a), neg2 = splat2(-mn);
+#if SPEC_SCALAR_ACC
+  float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) {
+    const float2 e0 = ex2_pair(__ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), a2, neg2), i);
+    const float2 e1 = ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1);
+    t0 += e0.x; t1 += e0.y; t2 += e1.x; t3 += e1.y;
+  }
+  z += (t0 + t1) + (t2 + t3);
+#else
   float2 s0 = splat2(0.f), s1 = splat2(0.f);
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
@@ -293,6 +340,7 @@ __device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid,
     s1 = __fadd2_rn(s1, ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1));
   }
   z += (s0.x + s0.y) + (s1.x + s1.y);
+#endif
 }
 
 // Pass 2: probabilities of 32 query rows for this thread's key, reduced into acc (two packed
@@ -309,8 +357,12 @@ __device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const f
       acc[0] = make_float2(fmaxf(acc[0].x, p0.x), fmaxf(acc[0].y, p0.y));
       acc[1] = make_float2(fmaxf(acc[1].x, p1.x), fmaxf(acc[1].y, p1.y));
     } else {
+#if SPEC_SCALAR_ACC
+      acc[0].x += p0.x; acc[0].y += p0.y; acc[1].x += p1.x; acc[1].y += p1.y;
+#else
       acc[0] = __fadd2_rn(acc[0], p0);
       acc[1] = __fadd2_rn(acc[1], p1);
+#endif
     }
   }
 }
@@ -558,7 +610,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
             const float* negc = c_sm + ch * 128 + half * hw;
             tmem_ld32(taddr, ra);
-            if (kLoadAhead) {
+            if (kLoadAhead2) {
               if (hw > 32) tmem_ld32(taddr + 32, rb);
               tmem_ld_wait(ra);
               if (hw > 32) tmem_ld_wait(rb);
@@ -573,7 +625,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);
-            if (kLoadAhead) {
+            if (kLoadAhead2) {
               prob_accumulate<MAXRED>(ra, negc, a2, acc);
               if (hw > 32) prob_accumulate<MAXRED>(rb, negc + 32, a2, acc);
             } else {
