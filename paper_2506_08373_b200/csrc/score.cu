@@ -55,7 +55,6 @@ constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32
 constexpr bool kLoadAhead = SPEC_LOAD_AHEAD;    // pass 1: fetch a work item's second 32 columns before the math on the first
 constexpr bool kLoadAhead2 = SPEC_LOAD_AHEAD2;  // pass 2: the same
 constexpr int kBufCols = 128;
-constexpr int kNumBufs = 4;
 constexpr int kTileKeys = 128;
 constexpr int kMaxStages = 8;
 constexpr int kMaxMTiles = 10;
@@ -374,7 +373,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr int BUFCOLS = kBufCols;
-  constexpr int NBUF = kNumBufs;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint8_t* k_sm = smem;
@@ -402,11 +400,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
   }
   if (tid == 32) {
-    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 2); }   // both MMA threads release a stage
+    // pass 1: one MMA thread, every buffer drained by all 16 epilogue warps;
+    // pass 2: two MMA threads release a stage, a buffer is drained by the 8 warps of one pair
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], PASS == 1 ? 1 : 2); }
     mbar_init(q_full, 1);
-    mbar_init(q_empty, 2);
-    // a buffer is drained by the eight warps of one warpgroup pair
-    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 8); }
+    mbar_init(q_empty, PASS == 1 ? 1 : 2);
+    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], PASS == 1 ? 16 : 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -419,6 +418,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
   const uint32_t tmem_base = *tmem_slot;
   const int n_kh = p.d / 64;                               // 64-element halves of the contraction
   const uint32_t q_half_bytes = (uint32_t)p.M_pad * 128u;
+  // K ring: [64-element half of the contraction][stage][128 keys x 128 bytes], so that two
+  // consecutive stages form one 256-key operand
+  const uint32_t k_half_bytes = (uint32_t)p.n_stages * (128u * 128u);
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer ----
@@ -442,10 +444,18 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           ok = mbar_wait(&k_empty[stage], par ^ 1, abort_flag);
           if (!ok) break;
           mbar_expect_tx(&k_full[stage], p.stage_bytes);
-          uint8_t* dst = k_sm + (size_t)stage * p.stage_bytes;
+          uint8_t* dst = k_sm + (size_t)stage * (128 * 128);
           const int row = sg.begin + (sg.t0 + t) * kTileKeys;
           for (int kh = 0; kh < n_kh; ++kh)
-            tma_load_4d(dst + kh * (128 * 128), &tm_k, kh * 64, row, sg.h, sg.l, &k_full[stage]);
+            tma_load_4d(dst + kh * k_half_bytes, &tm_k, kh * 64, row, sg.h, sg.l, &k_full[stage]);
+        }
+        if (PASS == 1 && ok && (sg.nt & 1)) {
+          // pass 1 consumes stages in pairs: an odd segment is padded with an empty slot
+          const int stage = kit % p.n_stages;
+          ok = mbar_wait(&k_empty[stage], ((kit / p.n_stages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive(&k_full[stage]);
+          ++kit;
         }
       }
     }
@@ -461,56 +471,82 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
       const int strm = warp == 1 ? 0 : 1;
       SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
       Seg sg;
-      uint32_t kit = 0, bit = 0, nseg = 0, j = 0;            // j: items issued to my pair
+      uint32_t kit = 0, nseg = 0, j = 0;                    // j: items issued (pass 2: to my pair)
       bool ok = true;
       const uint32_t idesc_full = make_idesc(128);
       const uint32_t idesc_last = make_idesc(PASS == 1 ? 128 : p.cw_last);
       const int n_sub = PASS == 1 ? p.M_pad / 128 : p.n_chunks;
       const uint32_t q_lo0 = desc_lo(smem_u32(q_sm)), k_lo0 = desc_lo(smem_u32(k_sm));
       const uint32_t q_half16 = q_half_bytes >> 4;
-      while (ok && seg_next(it, p, tp, sg)) {
+      const uint32_t k_half16 = k_half_bytes >> 4;
+      while (ok && (PASS == 2 || strm == 0) && seg_next(it, p, tp, sg)) {
         ok = mbar_wait(q_full, nseg & 1, abort_flag);
         if (!ok) break;
         ++nseg;
         tc_fence_after();
-        for (int t = 0; t < sg.nt && ok; ++t, ++kit) {
-          const int stage = kit % p.n_stages;
-          ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t k_lo = k_lo0 + stage * (p.stage_bytes >> 4);
-          // Pass 1: the tile's blocks of 128 query rows alternate between the pairs (item b of
-          // the CTA goes to pair b % 2).  Pass 2: the whole tile, all chunks of query rows,
-          // belongs to the pair with the parity of the tile's index in the segment, so that a
-          // key is reduced by one pair only.
-          const bool whole_tile_mine = PASS == 2 && (t & 1) == strm;
-          if (PASS == 1 || whole_tile_mine) {
-            for (int sub = 0; sub < n_sub; ++sub, ++bit) {
-              if (PASS == 1 && (int)(bit & 1u) != strm) continue;
-              const int buf = strm + 2 * (int)(j & 1u);
+        if (PASS == 1) {
+          // Work item = (two key tiles, block of 128 query rows): D[128 x 256] in one of two
+          // 256-column buffers, drained by all epilogue warps.  Half as many instructions per
+          // logit as with 128-key items, so one issuing thread keeps ahead of the epilogue.
+          for (int t = 0; t < sg.nt && ok; t += 2, kit += 2) {
+            const int stage = kit % p.n_stages;              // even: n_stages is even and segments use whole pairs
+            const uint32_t par = (kit / p.n_stages) & 1;
+            ok = mbar_wait(&k_full[stage], par, abort_flag) && mbar_wait(&k_full[stage + 1], par, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t k_lo = k_lo0 + stage * ((128 * 128) >> 4);
+            const uint32_t idesc = t + 1 < sg.nt ? make_idesc(256) : idesc_full;   // the padding slot holds no keys
+            for (int sub = 0; sub < n_sub; ++sub, ++j) {
+              const int buf = (int)(j & 1u);
               ok = mbar_wait(&t_empty[buf], ((j >> 1) & 1) ^ 1, abort_flag);
               if (!ok) break;
-              ++j;
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
+              const uint32_t d_tmem = tmem_base + buf * 256;
               const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);      // 128 query rows of 128 bytes
-              const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
 #pragma unroll
               for (int kh = 0; kh < 2; ++kh) {
                 if (kh < n_kh) {
 #pragma unroll
-                  for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t qd = desc_at(q_lo + kh * q_half16 + ks * 2);
-                    const uint64_t kd = desc_at(k_lo + kh * ((128 * 128) >> 4) + ks * 2);
-                    if (PASS == 1) tc_mma(d_tmem, qd, kd, idesc, (kh | ks) != 0);
-                    else           tc_mma(d_tmem, kd, qd, idesc, (kh | ks) != 0);
-                  }
+                  for (int ks = 0; ks < 4; ++ks)
+                    tc_mma(d_tmem, desc_at(q_lo + kh * q_half16 + ks * 2), desc_at(k_lo + kh * k_half16 + ks * 2), idesc, (kh | ks) != 0);
                 }
               }
               tc_commit(&t_full[buf]);
             }
+            if (ok) { tc_commit(&k_empty[stage]); tc_commit(&k_empty[stage + 1]); }
           }
-          if (ok) tc_commit(&k_empty[stage]);        // arrives once my MMAs on this stage (if any) retire
+        } else {
+          // The whole tile, all chunks of query rows, belongs to the pair with the parity of the
+          // tile's index in the segment, so that a key is reduced by one pair only.
+          for (int t = 0; t < sg.nt && ok; ++t, ++kit) {
+            const int stage = kit % p.n_stages;
+            ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t k_lo = k_lo0 + stage * ((128 * 128) >> 4);
+            if ((t & 1) == strm) {
+              for (int sub = 0; sub < n_sub; ++sub) {
+                const int buf = strm + 2 * (int)(j & 1u);
+                ok = mbar_wait(&t_empty[buf], ((j >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                ++j;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
+                const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);
+                const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {
+                  if (kh < n_kh) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                      tc_mma(d_tmem, desc_at(k_lo + kh * k_half16 + ks * 2), desc_at(q_lo + kh * q_half16 + ks * 2), idesc, (kh | ks) != 0);
+                  }
+                }
+                tc_commit(&t_full[buf]);
+              }
+            }
+            if (ok) tc_commit(&k_empty[stage]);      // arrives once my MMAs on this stage (if any) retire
+          }
         }
         if (ok) tc_commit(q_empty);
       }
@@ -530,24 +566,24 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     bool ok = true;
     uint32_t ra[32], rb[32];
     if (PASS == 1) {
-      // Work item = one 128 x 128 logit tile (query rows on lanes); this warpgroup owns 64 of
-      // its key columns.
+      // Work item = 128 query rows (on lanes) x 256 keys (two tiles) in one of two 256-column
+      // buffers; every warpgroup owns 64 of its key columns.
       const int n_mt = p.M_pad / 128;
       float mrun[kMaxMTiles], zrun[kMaxMTiles];
       while (ok && seg_next(it, p, tp, sg)) {
 #pragma unroll
         for (int i = 0; i < kMaxMTiles; ++i) { mrun[i] = -INFINITY; zrun[i] = 0.f; }
-        for (int t = 0; t < sg.nt && ok; ++t) {
-          const int nvh = min(kTileKeys, sg.n - (sg.t0 + t) * kTileKeys) - half * 64;   // valid keys in my half
+        for (int t = 0; t < sg.nt && ok; t += 2) {
+          const int n_item = t + 1 < sg.nt ? 2 * kTileKeys : kTileKeys;            // the last item of an odd segment is one tile
+          const int nvh = min(n_item, sg.n - (sg.t0 + t) * kTileKeys) - wg * 64;   // valid keys in my 64 columns
           for (int mt = 0; mt < n_mt; ++mt, ++bit) {
-            if ((int)(bit & 1u) != pair) continue;
-            const int buf = bit % NBUF;
-            ok = mbar_wait(&t_full[buf], (bit / NBUF) & 1, abort_flag);
+            const int buf = (int)(bit & 1u);
+            ok = mbar_wait(&t_full[buf], (bit >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             float m = mrun[mt], z = zrun[mt];
             if (nvh > 0) {
-              const uint32_t taddr = lane_base + buf * BUFCOLS + half * 64;
+              const uint32_t taddr = lane_base + buf * 256 + wg * 64;
               tmem_ld32(taddr, ra);
               if (kLoadAhead) {
                 if (nvh > 32) tmem_ld32(taddr + 32, rb);
@@ -804,6 +840,7 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   const int smem_max = 227 * 1024;
   int stages = (smem_max - (int)p.q_bytes - small) / (int)p.stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  stages &= ~1;                                            // pass 1 consumes the ring two stages at a time
   if (stages < 2) return fail(SPEC_ERR_UNSUPPORTED, "not enough shared memory for two key stages (M=%d, head_dim=%d)", M, d);
   p.n_stages = stages;
   int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
