@@ -37,7 +37,10 @@ constexpr int kEpilogueThreads = kEpilogueWarpgroups * 128;
 constexpr int kMmaWarpB = 2 + kEpilogueThreads / 32;    // second MMA-issuing warp, after the epilogue warps
 constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_POLY_PAIRS
-#define SPEC_POLY_PAIRS 3
+#define SPEC_POLY_PAIRS 5
+#endif
+#ifndef SPEC_EX2_INPLACE
+#define SPEC_EX2_INPLACE 0
 #endif
 #ifndef SPEC_POLY_SCALAR
 #define SPEC_POLY_SCALAR 0
@@ -45,16 +48,8 @@ constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_SCALAR_ACC
 #define SPEC_SCALAR_ACC 0
 #endif
-#ifndef SPEC_LOAD_AHEAD
-#define SPEC_LOAD_AHEAD 0
-#endif
 constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes
-#ifndef SPEC_LOAD_AHEAD2
-#define SPEC_LOAD_AHEAD2 0
-#endif
-constexpr bool kLoadAhead = SPEC_LOAD_AHEAD;    // pass 1: fetch a work item's second 32 columns before the math on the first
-constexpr bool kLoadAhead2 = SPEC_LOAD_AHEAD2;  // pass 2: the same
-constexpr int kBufCols = 128;
+constexpr int kBufCols = 128;                 // TMEM columns of a pass-2 accumulator buffer (pass 1 uses two of 256)
 constexpr int kTileKeys = 128;
 constexpr int kMaxStages = 8;
 constexpr int kMaxMTiles = 10;
@@ -152,27 +147,18 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane.
+// 32 consecutive fp32 columns of this thread's TMEM lane, complete on return (the load and
+// the wait for it are one statement, so no use of the registers can be scheduled in between).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-}
-// Completes all earlier tcgen05.ld of this thread; the registers are tied to the wait so that
-// no use of them can be scheduled above it.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-      :: "memory");
+      : "r"(taddr) : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -266,7 +252,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 // 2^x for both lanes on the MUFU unit.
-__device__ __forceinline__ float2 ex2_mufu2(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+__device__ __forceinline__ float2 ex2_mufu2(float2 x) {
+#if SPEC_EX2_INPLACE
+  // in place, so that the two results stay in the register pair the packed add reads
+  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(x.x));
+  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(x.y));
+  return x;
+#else
+  return make_float2(ex2(x.x), ex2(x.y));
+#endif
+}
 // 2^x for both lanes without the MUFU unit: x = n + f with n = round(x), |f| <= 1/2 (adding
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic with relative error 7.5e-5,
 // then n is added into the exponent field.  x is clamped at -125 so the exponent cannot wrap.
@@ -564,7 +559,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     Seg sg;
     uint32_t bit = 0;
     bool ok = true;
-    uint32_t ra[32], rb[32];
+    uint32_t ra[32];
     if (PASS == 1) {
       // Work item = 128 query rows (on lanes) x 256 keys (two tiles) in one of two 256-column
       // buffers; every warpgroup owns 64 of its key columns.
@@ -585,28 +580,13 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (nvh > 0) {
               const uint32_t taddr = lane_base + buf * 256 + wg * 64;
               tmem_ld32(taddr, ra);
-              if (kLoadAhead) {
-                if (nvh > 32) tmem_ld32(taddr + 32, rb);
-                tmem_ld_wait(ra);
-                if (nvh > 32) tmem_ld_wait(rb);
-              } else {
-                tmem_ld_wait(ra);
-                if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z);
-                if (nvh > 32) {
-                  tmem_ld32(taddr + 32, ra);
-                  tmem_ld_wait(ra);
-                }
-              }
+              if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z);
+              if (nvh > 32) tmem_ld32(taddr + 32, ra);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);       // all reads done: the buffer can be refilled
-            if (kLoadAhead) {
-              if (nvh > 0) { if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z); }
-              if (nvh >= 64) stats_update<false>(rb, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(rb, nvh - 32, p.a, m, z);
-            } else {
-              if (nvh >= 64) stats_update<false>(ra, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(ra, nvh - 32, p.a, m, z);
-            }
+            if (nvh >= 64) stats_update<false>(ra, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(ra, nvh - 32, p.a, m, z);
             mrun[mt] = m;
             zrun[mt] = z;
           }
@@ -646,27 +626,14 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
             const float* negc = c_sm + ch * 128 + half * hw;
             tmem_ld32(taddr, ra);
-            if (kLoadAhead2) {
-              if (hw > 32) tmem_ld32(taddr + 32, rb);
-              tmem_ld_wait(ra);
-              if (hw > 32) tmem_ld_wait(rb);
-            } else {
-              tmem_ld_wait(ra);
-              if (hw > 32) {
-                prob_accumulate<MAXRED>(ra, negc, a2, acc);
-                tmem_ld32(taddr + 32, ra);
-                tmem_ld_wait(ra);
-              }
+            if (hw > 32) {
+              prob_accumulate<MAXRED>(ra, negc, a2, acc);
+              tmem_ld32(taddr + 32, ra);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);
-            if (kLoadAhead2) {
-              prob_accumulate<MAXRED>(ra, negc, a2, acc);
-              if (hw > 32) prob_accumulate<MAXRED>(rb, negc + 32, a2, acc);
-            } else {
-              prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
-            }
+            prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
           }
           if (!ok) break;
           const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
