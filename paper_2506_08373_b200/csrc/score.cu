@@ -69,6 +69,7 @@ struct ScoreParams {
   int32_t* status;
   long long T;
   int n_in, n_seq, L, Hq, Hkv, G, R, M, M_pad, d;
+  int causal, n_window;  // causal != 0: window row r sees keys up to position n - n_window + r only
   int n_stages, n_chunks, cw_last;   // pass 2: chunks of 128 query rows, the last of cw_last (64 or 128)
   int reduce;
   float a;              // softmax_scale * log2(e)
@@ -351,13 +352,26 @@ __device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const f
       acc[0] = make_float2(fmaxf(acc[0].x, p0.x), fmaxf(acc[0].y, p0.y));
       acc[1] = make_float2(fmaxf(acc[1].x, p1.x), fmaxf(acc[1].y, p1.y));
     } else {
-#if SPEC_SCALAR_ACC
-      acc[0].x += p0.x; acc[0].y += p0.y; acc[1].x += p1.x; acc[1].y += p1.y;
-#else
       acc[0] = __fadd2_rn(acc[0], p0);
       acc[1] = __fadd2_rn(acc[1], p1);
-#endif
     }
+  }
+}
+
+// The same for a key tile that reaches into the causal window: the probability of query row
+// (row0 + i) for this thread's key (position `key` of a sequence of n) is dropped when the row
+// is window row r < n_window and the key lies after the row's own position n - n_window + r.
+// Plain scalar code: only the last tile or two of a sequence come here.
+template <bool MAXRED>
+__device__ __forceinline__ void prob_accumulate_causal(const uint32_t (&r)[32], const float* __restrict__ negc, float a,
+                                                       float2 (&acc)[2], int row0, int R, int n_window, int n, int key) {
+  int rr = row0 % R;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float pr = ex2(fmaf(__uint_as_float(r[i]), a, negc[i]));
+    if (rr < n_window && key > max(n - n_window + rr, 0)) pr = 0.f;
+    if (MAXRED) acc[0].x = fmaxf(acc[0].x, pr); else acc[0].x += pr;
+    if (++rr == R) rr = 0;
   }
 }
 
@@ -570,23 +584,37 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         for (int i = 0; i < kMaxMTiles; ++i) { mrun[i] = -INFINITY; zrun[i] = 0.f; }
         for (int t = 0; t < sg.nt && ok; t += 2) {
           const int n_item = t + 1 < sg.nt ? 2 * kTileKeys : kTileKeys;            // the last item of an odd segment is one tile
-          const int nvh = min(n_item, sg.n - (sg.t0 + t) * kTileKeys) - wg * 64;   // valid keys in my 64 columns
+          const int key0 = (sg.t0 + t) * kTileKeys;                                // first key of the item
+          const int nvh = min(n_item, sg.n - key0) - wg * 64;                      // valid keys in my 64 columns
           for (int mt = 0; mt < n_mt; ++mt, ++bit) {
             const int buf = (int)(bit & 1u);
             ok = mbar_wait(&t_full[buf], (bit >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             float m = mrun[mt], z = zrun[mt];
+            int vis2 = 0;                                    // visible keys of the second 32 columns
             if (nvh > 0) {
               const uint32_t taddr = lane_base + buf * 256 + wg * 64;
+              // keys of my 64 columns that this thread's row may see
+              int vis = nvh;
+              const bool in_window = p.causal && key0 + n_item > sg.n - p.n_window;   // warp-uniform
+              if (in_window) {
+                const int rr = (mt * 128 + row_in_tile) % p.R;
+                if (rr < p.n_window) vis = min(nvh, max(sg.n - p.n_window + rr, 0) + 1 - (key0 + wg * 64));
+              }
               tmem_ld32(taddr, ra);
-              if (nvh >= 32) stats_update<false>(ra, 32, p.a, m, z); else stats_update<true>(ra, nvh, p.a, m, z);
+              if (!in_window && nvh >= 32) stats_update<false>(ra, 32, p.a, m, z);
+              else if (vis > 0) stats_update<true>(ra, min(vis, 32), p.a, m, z);
               if (nvh > 32) tmem_ld32(taddr + 32, ra);
+              vis2 = in_window || nvh < 64 ? vis - 32 : 32;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);       // all reads done: the buffer can be refilled
-            if (nvh >= 64) stats_update<false>(ra, 32, p.a, m, z); else if (nvh > 32) stats_update<true>(ra, nvh - 32, p.a, m, z);
+            if (nvh > 32) {
+              if (vis2 >= 32 && nvh >= 64) stats_update<false>(ra, 32, p.a, m, z);
+              else if (vis2 > 0) stats_update<true>(ra, min(vis2, 32), p.a, m, z);
+            }
             mrun[mt] = m;
             zrun[mt] = z;
           }
@@ -617,6 +645,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         float* out = p.scores + ((long long)sg.l * p.Hkv + sg.h) * p.T + sg.begin;
         for (int t = pair; t < sg.nt && ok; t += 2) {
           float2 acc[2] = {splat2(0.f), splat2(0.f)};
+          const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
+          const bool in_window = p.causal && (sg.t0 + t + 1) * kTileKeys > sg.n - p.n_window;   // warp-uniform
           for (int ch = 0; ch < p.n_chunks; ++ch, ++j) {
             const int buf = pair + 2 * (int)(j & 1u);
             ok = mbar_wait(&t_full[buf], (j >> 1) & 1, abort_flag);
@@ -625,18 +655,20 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const int hw = (ch == p.n_chunks - 1 ? p.cw_last : 128) >> 1;     // my columns: 32 or 64
             const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
             const float* negc = c_sm + ch * 128 + half * hw;
+            const int row0 = ch * 128 + half * hw;              // query row of my first column
             tmem_ld32(taddr, ra);
             if (hw > 32) {
-              prob_accumulate<MAXRED>(ra, negc, a2, acc);
+              if (!in_window) prob_accumulate<MAXRED>(ra, negc, a2, acc);
+              else prob_accumulate_causal<MAXRED>(ra, negc, p.a, acc, row0, p.R, p.n_window, sg.n, key);
               tmem_ld32(taddr + 32, ra);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&t_empty[buf]);
-            prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
+            if (!in_window) prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
+            else prob_accumulate_causal<MAXRED>(ra, hw > 32 ? negc + 32 : negc, p.a, acc, hw > 32 ? row0 + 32 : row0, p.R, p.n_window, sg.n, key);
           }
           if (!ok) break;
-          const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
           if (key < sg.n) {
             // The output was zero-filled; the two warpgroups of the pair contribute once per key.
             const float v0 = acc[0].x, v1 = acc[0].y, v2 = acc[1].x, v3 = acc[1].y;
@@ -739,7 +771,7 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   if (rc != SPEC_OK) return rc;
   if (!q || !k || !scores_out) return fail(SPEC_ERR_BAD_ARG, "q, k and scores_out must not be NULL");
   if (reduce != SPEC_REDUCE_SUM && reduce != SPEC_REDUCE_MAX) return fail(SPEC_ERR_BAD_ARG, "reduce=%d is not a spec_reduce value", reduce);
-  if (causal_window != 0) return fail(SPEC_ERR_NOT_IMPLEMENTED, "causal_window=1 is not implemented yet");
+  if (causal_window != 0 && causal_window != 1) return fail(SPEC_ERR_BAD_ARG, "causal_window=%d must be 0 or 1", causal_window);
   if (!(pr->softmax_scale > 0.f) || !(pr->softmax_scale < 1e30f)) return fail(SPEC_ERR_BAD_ARG, "softmax_scale must be positive and finite");
   if (!aligned16(q) || !aligned16(k)) return fail(SPEC_ERR_ALIGNMENT, "q and k must be 16-byte aligned");
   const int d = pr->head_dim;
@@ -800,6 +832,8 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   p.n_chunks = (M64 + 127) / 128;
   p.cw_last = M64 - (p.n_chunks - 1) * 128;
   p.reduce = reduce;
+  p.causal = causal_window;
+  p.n_window = pr->n_window;
   p.a = (float)((double)pr->softmax_scale * 1.4426950408889634);
   p.q_bytes = (uint32_t)M_pad * d * 2;
   p.stage_bytes = (uint32_t)kTileKeys * d * 2;

@@ -102,6 +102,26 @@ def test_score_max_reduce_and_row_weights(B, W, oracle):
     assert got.max() <= 1.0 + 1e-5
 
 
+def test_score_causal_window(B, W, oracle):
+    """Window row r sees keys up to its own prompt position only (the model's causal mask)."""
+    cases = [small(W, n_in=600), small(W, n_in=257, n_window=40, n_lookahead=3),
+             small(W, n_in=20, n_window=32, n_lookahead=5),            # window longer than the prompt
+             W.CONFIGS[4].replace(n_layers=1, n_seq=5, len_lo=1, len_hi=700, c_max=16)]
+    for w in cases:
+        g = Gpu(B, W, w, [0])
+        for reduce in (B.REDUCE_SUM, B.REDUCE_MAX):
+            got = g.score(reduce=reduce, causal_window=1).cpu().numpy()
+            ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale, mode=reduce,
+                                    causal_window=True)
+            assert_scores_close(got, ref, g.cu)
+    # the mask changes the result where it should
+    w = cases[0]
+    g = Gpu(B, W, w, [0])
+    a, b = g.score(causal_window=0), g.score(causal_window=1)
+    assert not torch.equal(a[..., -w.n_window:], b[..., -w.n_window:])
+    assert torch.allclose(a.sum(-1), b.sum(-1), rtol=1e-4)              # rows still sum to one
+
+
 def test_score_token_major_key_layout_and_reproducibility(B, W, oracle):
     w = small(W, n_in=900)
     g = Gpu(B, W, w, [0, 1])

@@ -32,10 +32,10 @@ class Gpu:
         self.ws = torch.empty(max(B.spec_workspace_bytes(self.pr), 16), dtype=torch.uint8, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    def score(self, reduce=0, row_weight=None):
+    def score(self, reduce=0, row_weight=None, causal_window=0):
         scores = torch.full((self.L, self.w.n_kv_heads, self.T), float("nan"), dtype=torch.float32, device="cuda")
         self.B.spec_score(self.pr, self.q, self.k, scores, self.ws, row_weight=row_weight, reduce=reduce,
-                          status_word=self.status)
+                          causal_window=causal_window, status_word=self.status)
         torch.cuda.synchronize()
         assert self.status.item() == 0
         return scores
