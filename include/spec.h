@@ -176,6 +176,29 @@ int32_t specpc_token_select(const spec_problem* problem, const float* scores, in
                             int32_t* status_word, void* stream);
 
 /*
+ * Prompt compression for the SpecKV-PC cascade -- Section 4.3 (SpecPC first cuts the prompt to
+ * the kept tokens, then SpecKV runs on the compressed prompt).
+ *
+ * Gathers, for every layer and KV head, the K (and V) rows of the tokens in `keep` and packs the
+ * sequences back to back: cu_seqlens_out[s] = n_keep[0] + ... + n_keep[s-1] is computed on the
+ * device, so no host synchronisation is needed between specpc_token_select and the SpecKV calls
+ * on the compressed prompt (pass cu_seqlens_out as the new problem's cu_seqlens, out_tokens as
+ * its total_tokens and keep_capacity as its n_in bound).
+ *
+ *  keep            [n_seq, keep_capacity] int32 sequence-local positions, ascending (entries
+ *                  beyond n_keep[s] are ignored)
+ *  n_keep          [n_seq] int32
+ *  k_out, v_out    [n_layers, n_kv_heads, out_tokens, head_dim] bf16; rows past the packed total
+ *                  are left untouched.  v and v_out may both be NULL
+ *  cu_seqlens_out  [n_seq + 1] int32, written by the call
+ * A position outside its sequence, n_keep outside [0, keep_capacity] or a packed total above
+ * out_tokens is skipped and reported as SPEC_ERR_BAD_ARG in status_word.
+ */
+int32_t spec_gather_tokens(const spec_problem* problem, const void* k, const void* v, const int32_t* keep,
+                           int32_t keep_capacity, const int32_t* n_keep, void* k_out, void* v_out,
+                           int32_t out_tokens, int32_t* cu_seqlens_out, int32_t* status_word, void* stream);
+
+/*
  * specpc_token_select for callers that cannot allocate device memory.
  *
  * (No counterpart in the paper: this is a packaging variant of the call above.)

@@ -141,6 +141,23 @@ def compact(src: np.ndarray, cu: Sequence[int], idx: np.ndarray, block_table: Op
     return dst
 
 
+def gather_tokens(src: np.ndarray, cu: Sequence[int], keep: np.ndarray, n_keep: np.ndarray, out_tokens: int):
+    """Prompt compression of the SpecKV-PC cascade (Section 4.3): the rows of the kept tokens of every
+    sequence, packed back to back.  src uint16 [L, Hkv, T, d]; keep int32 [n_seq, cap] sequence-local;
+    -> (dst uint16 [L, Hkv, out_tokens, d] with untouched rows 0xFFFF, cu_out int32 [n_seq + 1])."""
+    assert src.dtype == np.uint16
+    L, Hkv, T, d = src.shape
+    cu = _cu(cu)
+    n_seq = len(cu) - 1
+    dst = np.full((L, Hkv, out_tokens, d), 0xFFFF, dtype=np.uint16)
+    cu_out = np.zeros(n_seq + 1, dtype=np.int32)
+    for s in range(n_seq):
+        cu_out[s + 1] = cu_out[s] + int(n_keep[s])
+        for c in range(int(n_keep[s])):
+            dst[:, :, cu_out[s] + c, :] = src[:, :, cu[s] + int(keep[s, c]), :]
+    return dst, cu_out
+
+
 def specpc_select(scores: np.ndarray, cu: Sequence[int], reduce: int, pool_kind: int, k: int, c_max: int,
                   n_neighbor: int, n_forced_tail: int = 0, keep_capacity: Optional[int] = None):
     """scores float64 [L, Hkv, T] -> (keep int32 [n_seq, cap] (-1 padded), n_keep [n_seq],

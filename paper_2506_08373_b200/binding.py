@@ -18,7 +18,7 @@ REDUCE_SUM, REDUCE_MAX = 0, 1
 POOL_MAX, POOL_AVG = 0, 1
 
 EXPORTS = ("spec_workspace_bytes", "spec_last_error", "spec_score", "spec_pool_topk", "spec_compact_kv",
-           "specpc_token_select", "specpc_token_select_static")
+           "specpc_token_select", "spec_gather_tokens", "specpc_token_select_static")
 STATIC_MAX_TOKENS = 262144
 
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.spec_compact_kv.argtypes = [pp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp]
         L.specpc_token_select.restype = i32
         L.specpc_token_select.argtypes = [pp, vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, sz, vp, vp]
+        L.spec_gather_tokens.restype = i32
+        L.spec_gather_tokens.argtypes = [pp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp]
         L.specpc_token_select_static.restype = i32
         L.specpc_token_select_static.argtypes = [pp, vp, i32, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
         _lib = L
@@ -145,6 +147,13 @@ def specpc_token_select(problem, scores, layer_head_reduce, pool, pool_k, c_max,
                                      n_neighbor, n_forced_tail, _ptr(keep_out), keep_capacity, _ptr(n_keep_out),
                                      _ptr(workspace), workspace.numel() * workspace.element_size(),
                                      _ptr(status_word), _stream()))
+
+
+def spec_gather_tokens(problem, k, v, keep, keep_capacity, n_keep, k_out, v_out, out_tokens, cu_seqlens_out,
+                       status_word=None):
+    _check(lib().spec_gather_tokens(ctypes.byref(problem), _ptr(k), _ptr(v), _ptr(keep), keep_capacity, _ptr(n_keep),
+                                    _ptr(k_out), _ptr(v_out), out_tokens, _ptr(cu_seqlens_out), _ptr(status_word),
+                                    _stream()))
 
 
 def specpc_token_select_static(problem, scores, layer_head_reduce, pool, pool_k, c_max, n_neighbor, n_forced_tail,

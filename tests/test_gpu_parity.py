@@ -411,3 +411,108 @@ def test_specpc_config3_full(B, W, oracle):
     near = np.flatnonzero(np.abs(tok - th[0]) <= band)
     for j in set(got) ^ ref_keep:
         assert np.any(np.abs(near - j) <= w.n_neighbor), "keep-list difference at %d outside the band" % j
+
+
+# ------------------------------------------------------------------ widening rows -----
+
+def test_vertical_indices_are_a_second_top_k(B, W, oracle):
+    """Algorithm 1 line 11: i_vert = topk(s, n_vert) on the same pooled scores as i_cache (line 13) is the
+    same call with another budget; the smaller set is contained in the larger one."""
+    w = small(W, n_in=5000, c_max=256)
+    g = Gpu(B, W, w, [0, 1])
+    scores = g.score()
+    sc = scores.cpu().numpy().astype(np.float64)
+    i_cache, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 256, forced=w.n_window)
+    i_vert, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 1024)
+    o_vert, _, _, _ = oracle.pool_topk(sc, g.cu, oracle.POOL_MAX, w.pool_k, 1024)
+    np.testing.assert_array_equal(i_vert.cpu().numpy(), o_vert)
+    small_set, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 256)
+    for l in range(2):
+        for h in range(w.n_kv_heads):
+            assert set(small_set[0, l, h].tolist()) <= set(i_vert[0, l, h].tolist())
+    assert i_cache.shape[-1] == 256
+
+
+def test_gather_tokens_bit_exact(B, W, oracle):
+    rng = np.random.default_rng(9)
+    L, H, d, cap = 2, 3, 128, 50
+    cu = [0, 300, 300, 1000]
+    T = 1000
+    k = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
+    v = torch.from_numpy(rng.integers(-32768, 32767, size=(L, H, T, d)).astype(np.int16)).view(torch.bfloat16).cuda()
+    n_keep = np.array([37, 0, 50], dtype=np.int32)
+    keep = np.full((3, cap), -1, dtype=np.int32)
+    for s, n in enumerate((300, 0, 700)):
+        keep[s, :n_keep[s]] = np.sort(rng.choice(max(n, 1), n_keep[s], replace=False)) if n_keep[s] else []
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda")
+    pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=d, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=T, n_in=700, n_seq=3, cu_seqlens=cu_t, k=k, v=v)
+    out_tokens = 100
+    ko = torch.from_numpy(np.full((L, H, out_tokens, d), -1, np.int16)).view(torch.bfloat16).cuda()
+    vo = ko.clone()
+    cu_out = torch.full((4,), -9, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.spec_gather_tokens(pr, k, v, torch.from_numpy(keep).cuda(), cap, torch.from_numpy(n_keep).cuda(), ko, vo,
+                         out_tokens, cu_out, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for src, got in ((k, ko), (v, vo)):
+        want, want_cu = oracle.gather_tokens(bits(src), cu, keep, n_keep, out_tokens)
+        np.testing.assert_array_equal(bits(got), want)
+        np.testing.assert_array_equal(cu_out.cpu().numpy(), want_cu)
+    # a packed total beyond out_tokens is reported, nothing is written out of bounds
+    B.spec_gather_tokens(pr, k, None, torch.from_numpy(keep).cuda(), cap, torch.from_numpy(n_keep).cuda(), ko, None,
+                         60, cu_out, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == B.ERR_BAD_ARG
+
+
+def test_speckv_pc_cascade_without_host_sync(B, W, oracle):
+    """Section 4.3: SpecPC keep set from draft scores -> compressed target K/V -> SpecKV on the compressed
+    prompt, every length staying on the device.  Checked against the same chain of oracle functions."""
+    wd = W.CONFIGS[3].replace(n_in=3000, n_layers=2, c_max=200, n_planted=8)          # draft model
+    wt = small(W, n_in=3000, n_layers=2, c_max=64, seed=31)                              # target model
+    gd, gt = Gpu(B, W, wd, [0, 1]), Gpu(B, W, wt, [0, 1])
+    n, cap = 3000, 200 * 17
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # 1. SpecPC on the draft
+    sd = gd.score()
+    keep = torch.empty((1, cap), dtype=torch.int32, device="cuda")
+    n_keep = torch.empty((1,), dtype=torch.int32, device="cuda")
+    B.specpc_token_select(gd.pr, sd, B.REDUCE_SUM, B.POOL_MAX, 7, 200, 8, wd.n_window, keep, cap, n_keep, gd.ws,
+                          status_word=status)
+    # 2. compress the target's K/V (lengths stay on the device)
+    v = torch.randn(gt.k.shape, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).cuda()
+    gt.pr = B.make_problem(n_layers=2, n_q_heads=wt.n_q_heads, n_kv_heads=wt.n_kv_heads, head_dim=wt.head_dim,
+                           n_lookahead=wt.n_lookahead, n_window=wt.n_window, softmax_scale=wt.scale,
+                           total_tokens=n, n_in=n, k=gt.k, v=v)
+    kc = torch.zeros((2, wt.n_kv_heads, cap, wt.head_dim), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    cu2 = torch.empty((2,), dtype=torch.int32, device="cuda")
+    B.spec_gather_tokens(gt.pr, gt.k, v, keep, cap, n_keep, kc, vc, cap, cu2, status_word=status)
+    # 3. SpecKV on the compressed prompt
+    pr2 = B.make_problem(n_layers=2, n_q_heads=wt.n_q_heads, n_kv_heads=wt.n_kv_heads, head_dim=wt.head_dim,
+                         n_lookahead=wt.n_lookahead, n_window=wt.n_window, softmax_scale=wt.scale,
+                         total_tokens=cap, n_in=cap, n_seq=1, cu_seqlens=cu2, k=kc, v=vc)
+    ws2 = torch.empty(B.spec_workspace_bytes(pr2), dtype=torch.uint8, device="cuda")
+    s2 = torch.empty((2, wt.n_kv_heads, cap), dtype=torch.float32, device="cuda")
+    idx = torch.empty((1, 2, wt.n_kv_heads, 64), dtype=torch.int32, device="cuda")
+    ko = torch.empty((1, 2, wt.n_kv_heads, 64, wt.head_dim), dtype=torch.bfloat16, device="cuda")
+    vo = torch.empty_like(ko)
+    B.spec_score(pr2, gt.q, kc, s2, ws2, status_word=status)
+    B.spec_pool_topk(pr2, s2, B.POOL_MAX, 7, 64, wt.n_window, idx, None, status_word=status)
+    B.spec_compact_kv(pr2, kc, vc, idx, 64, ko, vo, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    # oracle chain on the GPU's keep list (the keep list itself is covered by the SpecPC parity test)
+    nk = int(n_keep.item())
+    keep_h, cu2_h = keep.cpu().numpy(), [0, nk]
+    assert cu2.cpu().tolist() == cu2_h and wd.n_window <= nk <= cap
+    okc, _ = oracle.gather_tokens(bits(gt.k), [0, n], keep_h, np.array([nk], np.int32), cap)
+    np.testing.assert_array_equal(bits(kc)[:, :, :nk], okc[:, :, :nk])
+    ref = oracle.spec_score(bits(gt.q), okc[:, :, :nk].copy(), cu2_h, wt.n_lookahead, wt.n_window, wt.scale)
+    got = s2.cpu().numpy()[:, :, :nk]
+    assert_scores_close(got, ref, cu2_h)
+    oidx, _, _, _ = oracle.pool_topk(got.astype(np.float64), cu2_h, oracle.POOL_MAX, 7, 64, wt.n_window)
+    np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
+    np.testing.assert_array_equal(bits(ko), oracle.compact(okc[:, :, :nk].copy(), cu2_h, oidx))

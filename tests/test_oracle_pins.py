@@ -418,3 +418,18 @@ def test_config_geometry_matches_paper_constants():
     assert W.CONFIGS[3].n_window == int(vals["specpc_n_window"])
     lens = W.seq_lens(W.CONFIGS[4])
     assert len(lens) == 16 and min(lens) >= 4096 and max(lens) <= 65536
+
+
+def test_gather_tokens_is_fancy_indexing_packed(oracle):
+    """Prompt compression (Section 4.3): kept rows of every sequence, packed back to back."""
+    rng = np.random.default_rng(21)
+    L, H, d = 2, 3, 8
+    cu = [0, 5, 5, 17]
+    src = rng.integers(0, 65535, size=(L, H, 17, d)).astype(np.uint16)
+    keep = np.array([[0, 2, 4, -1], [-1, -1, -1, -1], [1, 3, 10, 11]], dtype=np.int32)
+    n_keep = np.array([3, 0, 4], dtype=np.int32)
+    dst, cu_out = oracle.gather_tokens(src, cu, keep, n_keep, 9)
+    assert list(cu_out) == [0, 3, 3, 7]
+    want = np.concatenate([src[:, :, [0, 2, 4], :], src[:, :, [6, 8, 15, 16], :]], axis=2)
+    np.testing.assert_array_equal(dst[:, :, :7], want)
+    assert (dst[:, :, 7:] == 0xFFFF).all()
