@@ -58,7 +58,11 @@ typedef enum {
 
 typedef enum {
   SPEC_POOL_MAX = 0,            /* hyper-parameter table: SpecKV pools with Max, k = 7 */
-  SPEC_POOL_AVG = 1             /* Algorithm 1 line 10 / Algorithm 2 line 8 as printed (AvgPool1D) */
+  SPEC_POOL_AVG = 1,            /* Algorithm 1 line 10 / Algorithm 2 line 8 as printed (AvgPool1D) */
+  SPEC_POOL_AVG_THEN_MAX = 2    /* specpc_token_select only: Algorithm 2 lines 8-9 in the printed order,
+                                   AvgPool1D(pool_k) then MaxPool1D(n_neighbor) BEFORE the selection, so
+                                   that exactly c_max tokens (plus the window) are kept; nothing is widened
+                                   afterwards */
 } spec_pool;
 
 /*
@@ -167,7 +171,8 @@ int32_t spec_compact_kv(const spec_problem* problem, const void* k, const void* 
  *  keep_out    [n_seq, keep_capacity] int32, ascending, padded with -1
  *  n_keep_out  [n_seq] int32
  * keep_capacity must be >= min(max_len, c_max*(2*n_neighbor+1) + n_forced_tail) where max_len is
- * n_in (cu_seqlens == NULL) or total_tokens; else SPEC_ERR_BAD_ARG.
+ * n_in (cu_seqlens == NULL) or total_tokens (with SPEC_POOL_AVG_THEN_MAX: min(max_len, c_max +
+ * n_forced_tail)); else SPEC_ERR_BAD_ARG.
  */
 int32_t specpc_token_select(const spec_problem* problem, const float* scores, int32_t layer_head_reduce,
                             int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,

@@ -21,7 +21,7 @@ _LIB = os.path.join(_DIR, "liboracle.so")
 _lib = None
 
 SUM, MAX = 0, 1          # reduction over query rows / over layers and heads
-POOL_MAX, POOL_AVG = 0, 1
+POOL_MAX, POOL_AVG, POOL_AVG_THEN_MAX = 0, 1, 2
 
 
 def build(force: bool = False) -> str:

@@ -271,7 +271,9 @@ int oracle_compact(const uint16_t* src, int64_t st_layer, int64_t st_head, int64
  *
  * Per sequence: t[j] = reduce over all (layer, KV head) of scores[l,h,cu[s]+j]
  * (reduce 0 = sum in (l, h) order, 1 = max; Algorithm 2 line 7 uses max), pool over
- * the eligible range [0, n - forced), keep the c_max best (Algorithm 2 line 10),
+ * the eligible range [0, n - forced) (pool 2: the printed order of Algorithm 2 lines
+ * 8-9, average pool of k then max pool of n_neighbor, and no widening below), keep
+ * the c_max best (Algorithm 2 line 10),
  * widen every kept position i to [i - n_neighbor, i + n_neighbor] clipped to the
  * eligible range, add the forced tail (the always-kept window), and return the
  * ascending list of distinct positions.
@@ -311,14 +313,26 @@ int oracle_specpc_select(const double* scores, int n_seq, const int32_t* cu, int
           }
         t[j] = a;
       }
-      oracle_pool(t, e, pool, k, pooled);
+      int widen = n_neighbor;
+      if (pool == 2) {
+        /* Algorithm 2 lines 8-9 in the printed order: AvgPool1D(k), then MaxPool1D(n_neighbor)
+         * before the selection; nothing is widened afterwards. */
+        double* avg = (double*)malloc(sizeof(double) * (size_t)e);
+        if (!avg) return -2;
+        oracle_pool(t, e, 1, k, avg);
+        oracle_pool(avg, e, 0, n_neighbor > 1 ? n_neighbor : 1, pooled);
+        free(avg);
+        widen = 0;
+      } else {
+        oracle_pool(t, e, pool, k, pooled);
+      }
       if (token_out) memcpy(token_out + b, pooled, sizeof(double) * (size_t)e);
       double th;
       const int n_top = select_top(pooled, e, c_max, top, &th);
       if (n_top < 0) return -2;
       if (thresh_out) thresh_out[s] = th;
       for (int c = 0; c < n_top; ++c) {
-        int lo = top[c] - n_neighbor, hi = top[c] + n_neighbor;
+        int lo = top[c] - widen, hi = top[c] + widen;
         if (lo < 0) lo = 0;
         if (hi > e - 1) hi = e - 1;
         for (int j = lo; j <= hi; ++j) mark[j] = 1;

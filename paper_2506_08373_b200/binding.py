@@ -15,7 +15,7 @@ SPEC_OK = 0
 ERR_BAD_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_IMPLEMENTED = \
     -1, -2, -3, -4, -5, -6, -7
 REDUCE_SUM, REDUCE_MAX = 0, 1
-POOL_MAX, POOL_AVG = 0, 1
+POOL_MAX, POOL_AVG, POOL_AVG_THEN_MAX = 0, 1, 2
 
 EXPORTS = ("spec_workspace_bytes", "spec_last_error", "spec_score", "spec_pool_topk", "spec_compact_kv",
            "specpc_token_select", "spec_gather_tokens", "specpc_token_select_static")

@@ -89,7 +89,7 @@ WorkspacePlan plan_workspace(const spec_problem* p) {
   w.rowc_bytes = (size_t)p->n_seq * p->n_layers * p->n_q_heads * (size_t)R * sizeof(float);
   off = align_up(off + w.rowc_bytes, 256);
   w.token_off = off;
-  w.token_bytes = (size_t)(p->total_tokens > 0 ? p->total_tokens : 1) * sizeof(float);
+  w.token_bytes = 2 * (size_t)(p->total_tokens > 0 ? p->total_tokens : 1) * sizeof(float);   // token scores, and their average pool
   off = align_up(off + w.token_bytes, 256);
   w.total = off;
   return w;

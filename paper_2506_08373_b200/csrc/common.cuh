@@ -33,7 +33,7 @@ struct WorkspacePlan {
   int score_ctas;          // persistent grid of the scoring kernels
   size_t partial_off, partial_bytes;   // per-segment row statistics (pass 1)
   size_t rowc_off, rowc_bytes;         // per-row softmax constants
-  size_t token_off, token_bytes;       // SpecPC token scores
+  size_t token_off, token_bytes;       // SpecPC token scores (two vectors of total_tokens floats)
   size_t total;
 };
 SPEC_HIDDEN WorkspacePlan plan_workspace(const spec_problem* p);

@@ -638,6 +638,19 @@ __global__ void __launch_bounds__(256) token_reduce_kernel(const float* __restri
   tok[t] = acc;
 }
 
+// First stage of Algorithm 2 lines 8-9 in the printed order: the average pool of the token
+// scores over each sequence's eligible range, written to a second vector.
+__global__ void __launch_bounds__(256) token_avgpool_kernel(const float* __restrict__ tok, float* __restrict__ out,
+                                                            const int32_t* __restrict__ cu, int n_in, int n_seq,
+                                                            int n_forced, int k) {
+  const int s = blockIdx.y;
+  int begin, n;
+  seq_range(cu, n_in, s, begin, n);
+  const int e = n - min(n_forced, n);
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < e; j += gridDim.x * blockDim.x)
+    out[begin + j] = pooled_at(tok + begin, e, j, SPEC_POOL_AVG, k);
+}
+
 struct KeepParams {
   const float* tok;
   const int32_t* cu;
@@ -748,8 +761,9 @@ static int select_smem_bytes(int max_len, int bitmap_words, int* cap_out) {
   return fixed + want * 4;
 }
 
-static int check_pool_args(int pool, int pool_k, int c_max, int n_forced_tail) {
-  if (pool != SPEC_POOL_MAX && pool != SPEC_POOL_AVG) return fail(SPEC_ERR_BAD_ARG, "pool=%d is not a spec_pool value", pool);
+static int check_pool_args(int pool, int pool_k, int c_max, int n_forced_tail, bool two_stage_ok = false) {
+  if (pool != SPEC_POOL_MAX && pool != SPEC_POOL_AVG && !(two_stage_ok && pool == SPEC_POOL_AVG_THEN_MAX))
+    return fail(SPEC_ERR_BAD_ARG, "pool=%d is not a spec_pool value this call accepts", pool);
   if (pool_k < 1 || pool_k > 255) return fail(SPEC_ERR_BAD_ARG, "pool_k=%d outside [1, 255]", pool_k);
   if (c_max < 1) return fail(SPEC_ERR_BAD_ARG, "c_max=%d must be >= 1", c_max);
   if (n_forced_tail < 0) return fail(SPEC_ERR_BAD_ARG, "n_forced_tail=%d is negative", n_forced_tail);
@@ -796,11 +810,13 @@ SPEC_EXPORT int32_t specpc_token_select(const spec_problem* pr, const float* sco
   if (!scores || !keep_out || !n_keep_out) return fail(SPEC_ERR_BAD_ARG, "scores, keep_out and n_keep_out must not be NULL");
   if (layer_head_reduce != SPEC_REDUCE_SUM && layer_head_reduce != SPEC_REDUCE_MAX)
     return fail(SPEC_ERR_BAD_ARG, "layer_head_reduce=%d is not a spec_reduce value", layer_head_reduce);
-  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);
+  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail, true);
   if (rc != SPEC_OK) return rc;
   if (n_neighbor < 0) return fail(SPEC_ERR_BAD_ARG, "n_neighbor=%d is negative", n_neighbor);
   const int max_len = max_seq_len(pr);
-  const int64_t worst = (int64_t)c_max * (2 * (int64_t)n_neighbor + 1) + n_forced_tail;
+  const bool two_stage = pool == SPEC_POOL_AVG_THEN_MAX;
+  if (two_stage && n_neighbor > 255) return fail(SPEC_ERR_BAD_ARG, "n_neighbor=%d as a pooling width exceeds 255", n_neighbor);
+  const int64_t worst = two_stage ? (int64_t)c_max + n_forced_tail : (int64_t)c_max * (2 * (int64_t)n_neighbor + 1) + n_forced_tail;
   const int64_t need_cap = worst < max_len ? worst : max_len;
   if (keep_capacity < need_cap)
     return fail(SPEC_ERR_BAD_ARG, "keep_capacity=%d is below the worst case %lld", keep_capacity, (long long)need_cap);
@@ -820,6 +836,18 @@ SPEC_EXPORT int32_t specpc_token_select(const spec_problem* pr, const float* sco
     token_reduce_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(scores, tok, T, pr->n_layers * pr->n_kv_heads,
                                                                      layer_head_reduce);
     SPEC_CUDA_OK(cudaGetLastError());
+  }
+  if (two_stage && T > 0) {
+    // Algorithm 2 lines 8-9 as printed: average pool, then the keep kernel max-pools with width
+    // n_neighbor before it selects, and widens nothing
+    float* tok2 = tok + T;
+    const dim3 grid((unsigned)((max_len + 255) / 256 > 0 ? (max_len + 255) / 256 : 1), (unsigned)pr->n_seq);
+    token_avgpool_kernel<<<grid, 256, 0, st>>>(tok, tok2, pr->cu_seqlens, pr->n_in, pr->n_seq, n_forced_tail, pool_k);
+    SPEC_CUDA_OK(cudaGetLastError());
+    tok = tok2;
+    pool = SPEC_POOL_MAX;
+    pool_k = n_neighbor > 1 ? n_neighbor : 1;
+    n_neighbor = 0;
   }
   KeepParams p;
   p.tok = tok; p.cu = pr->cu_seqlens; p.keep_out = keep_out; p.n_keep_out = n_keep_out;
@@ -880,7 +908,7 @@ SPEC_EXPORT int32_t specpc_token_select_static(const spec_problem* pr, const flo
   if (!scores || !keep_out || !n_keep_out) return fail(SPEC_ERR_BAD_ARG, "scores, keep_out and n_keep_out must not be NULL");
   if (layer_head_reduce != SPEC_REDUCE_SUM && layer_head_reduce != SPEC_REDUCE_MAX)
     return fail(SPEC_ERR_BAD_ARG, "layer_head_reduce=%d is not a spec_reduce value", layer_head_reduce);
-  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);
+  rc = check_pool_args(pool, pool_k, c_max, n_forced_tail);   // SPEC_POOL_AVG_THEN_MAX needs a second vector: not offered here
   if (rc != SPEC_OK) return rc;
   if (n_neighbor < 0) return fail(SPEC_ERR_BAD_ARG, "n_neighbor=%d is negative", n_neighbor);
   if (pr->total_tokens > SPEC_STATIC_MAX_TOKENS)

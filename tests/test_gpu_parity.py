@@ -388,6 +388,18 @@ def test_specpc_exact_on_dyadic_scores(B, W, oracle):
             ok, on, _, _ = oracle.specpc_select(scores.astype(np.float64), cu, reduce, 0, k, c_max, nb, forced, cap)
             np.testing.assert_array_equal(n_keep, on)
             np.testing.assert_array_equal(keep, ok)
+        # Algorithm 2 lines 8-9 in the printed order (average pool, max pool, then select): power-of-two
+        # pool widths keep the fp32 averages exact
+        for (c_max, nb, forced, k) in ((64, 8, 0, 4), (100, 1, 16, 8), (30, 5, 64, 1), (2000, 16, 0, 2)):
+            cap = 2095
+            keep, n_keep = run_keep(B, pr, st, reduce, B.POOL_AVG_THEN_MAX, k, c_max, nb, forced, cap, 4)
+            ok, on, _, _ = oracle.specpc_select(scores.astype(np.float64), cu, reduce, oracle.POOL_AVG_THEN_MAX, k,
+                                                c_max, nb, forced, cap)
+            np.testing.assert_array_equal(n_keep, on)
+            np.testing.assert_array_equal(keep, ok)
+            lens = np.diff(cu)
+            np.testing.assert_array_equal(n_keep, np.minimum(lens, np.minimum(c_max, np.maximum(lens - forced, 0))
+                                                             + np.minimum(forced, lens)))
 
 
 def test_specpc_config3_full(B, W, oracle):

@@ -433,3 +433,25 @@ def test_gather_tokens_is_fancy_indexing_packed(oracle):
     want = np.concatenate([src[:, :, [0, 2, 4], :], src[:, :, [6, 8, 15, 16], :]], axis=2)
     np.testing.assert_array_equal(dst[:, :, :7], want)
     assert (dst[:, :, 7:] == 0xFFFF).all()
+
+
+def test_specpc_printed_order_two_stage_pool(oracle):
+    """Algorithm 2 lines 8-10 as printed: AvgPool1D(k), MaxPool1D(n_neighbor), top-C_max union window, so
+    exactly C_max + n_window tokens survive; checked against the two pooling steps done by hand."""
+    rng = np.random.default_rng(33)
+    L, H, n, k, nb, c_max, win = 3, 2, 200, 5, 7, 20, 6
+    scores = rng.random((L, H, n))
+    keep, n_keep, tok, th = oracle.specpc_select(scores, [0, n], oracle.MAX, oracle.POOL_AVG_THEN_MAX, k, c_max, nb, win)
+    e = n - win
+    t = scores.max(axis=(0, 1))[:e]
+    avg = np.array([t[max(0, j - k // 2): min(e, j - k // 2 + k)].sum() / k for j in range(e)])
+    mx = np.array([avg[max(0, j - nb // 2): min(e, j - nb // 2 + nb)].max() for j in range(e)])
+    np.testing.assert_allclose(tok[:e], mx, rtol=1e-12)
+    order = sorted(range(e), key=lambda j: (-mx[j], j))[:c_max]
+    want = sorted(order) + list(range(e, n))
+    assert n_keep[0] == c_max + win
+    assert keep[0, :n_keep[0]].tolist() == want
+    # widths of one reduce it to the plain selection
+    k1, n1, _, _ = oracle.specpc_select(scores, [0, n], oracle.MAX, oracle.POOL_AVG_THEN_MAX, 1, c_max, 1, win)
+    k2, n2, _, _ = oracle.specpc_select(scores, [0, n], oracle.MAX, oracle.POOL_MAX, 1, c_max, 0, win)
+    np.testing.assert_array_equal(k1, k2)
