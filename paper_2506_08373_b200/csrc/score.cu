@@ -39,15 +39,6 @@ constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_POLY_PAIRS
 #define SPEC_POLY_PAIRS 5
 #endif
-#ifndef SPEC_EX2_INPLACE
-#define SPEC_EX2_INPLACE 0
-#endif
-#ifndef SPEC_POLY_SCALAR
-#define SPEC_POLY_SCALAR 0
-#endif
-#ifndef SPEC_SCALAR_ACC
-#define SPEC_SCALAR_ACC 0
-#endif
 constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes
 constexpr int kBufCols = 128;                 // TMEM columns of a pass-2 accumulator buffer (pass 1 uses two of 256)
 constexpr int kTileKeys = 128;
@@ -254,33 +245,12 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 
 // 2^x for both lanes on the MUFU unit.
 __device__ __forceinline__ float2 ex2_mufu2(float2 x) {
-#if SPEC_EX2_INPLACE
-  // in place, so that the two results stay in the register pair the packed add reads
-  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(x.x));
-  asm("ex2.approx.ftz.f32 %0, %0;" : "+f"(x.y));
-  return x;
-#else
   return make_float2(ex2(x.x), ex2(x.y));
-#endif
 }
 // 2^x for both lanes without the MUFU unit: x = n + f with n = round(x), |f| <= 1/2 (adding
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic with relative error 7.5e-5,
 // then n is added into the exponent field.  x is clamped at -125 so the exponent cannot wrap.
 __device__ __forceinline__ float2 ex2_poly2(float2 x) {
-#if SPEC_POLY_SCALAR
-  // range reduction packed, polynomial per lane: scalar FFMA takes its coefficients as immediates,
-  // the packed form needs every constant pair in registers
-  x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
-  const float2 big = splat2(12582912.f), minus1 = splat2(-1.f);
-  const float2 xr = __fadd2_rn(x, big);
-  const float2 n = __ffma2_rn(big, minus1, xr);
-  const float2 f = __ffma2_rn(n, minus1, x);
-  float q0 = fmaf(f.x, 0.0551713221f, 0.2426105440f), q1 = fmaf(f.y, 0.0551713221f, 0.2426105440f);
-  q0 = fmaf(q0, f.x, 0.6932609677f); q1 = fmaf(q1, f.y, 0.6932609677f);
-  q0 = fmaf(q0, f.x, 0.9999281168f); q1 = fmaf(q1, f.y, 0.9999281168f);
-  return make_float2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(xr.x) << 23)),
-                     __uint_as_float(__float_as_uint(q1) + (__float_as_uint(xr.y) << 23)));
-#else
   x = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
   const float2 xr = __fadd2_rn(x, splat2(12582912.f));
   const float2 n = __fadd2_rn(xr, splat2(-12582912.f));
@@ -290,7 +260,6 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
   q = __ffma2_rn(q, f, splat2(0.9999281168f));
   return make_float2(__uint_as_float(__float_as_uint(q.x) + (__float_as_uint(xr.x) << 23)),
                      __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(xr.y) << 23)));
-#endif
 }
 // Pair i (0..15) of a 32-element block: kPolyPairs of them, evenly spread, avoid the MUFU unit.
 __device__ __forceinline__ constexpr bool poly_pair(int i) {
@@ -318,16 +287,6 @@ __device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid,
   z *= ex2(m - mn);                                        // first block: 0 * 2^-inf = 0
   m = mn;
   const float2 a2 = splat2(a), neg2 = splat2(-mn);
-#if SPEC_SCALAR_ACC
-  float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
-#pragma unroll
-  for (int i = 0; i < 16; i += 2) {
-    const float2 e0 = ex2_pair(__ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), a2, neg2), i);
-    const float2 e1 = ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1);
-    t0 += e0.x; t1 += e0.y; t2 += e1.x; t3 += e1.y;
-  }
-  z += (t0 + t1) + (t2 + t3);
-#else
   float2 s0 = splat2(0.f), s1 = splat2(0.f);
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
@@ -335,7 +294,6 @@ __device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid,
     s1 = __fadd2_rn(s1, ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1));
   }
   z += (s0.x + s0.y) + (s1.x + s1.y);
-#endif
 }
 
 // Pass 2: probabilities of 32 query rows for this thread's key, reduced into acc (two packed

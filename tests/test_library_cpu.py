@@ -80,6 +80,17 @@ def test_bad_call_arguments_are_rejected_on_the_host(B):
     assert L.specpc_token_select(ctypes.byref(pr), one, 0, 0, 7, 16, 8, 0, one, 100, one, one, 1 << 30,
                                  None, None) == B.ERR_BAD_ARG
     assert "keep_capacity" in B.spec_last_error()
+    # the two-stage pool of Algorithm 2 is a SpecPC option only, and its keep list is exactly c_max + window
+    assert L.spec_pool_topk(ctypes.byref(pr), one, 2, 7, 16, 0, one, None, None, 0, None, None) == B.ERR_BAD_ARG
+    assert L.specpc_token_select(ctypes.byref(pr), one, 1, 2, 7, 16, 8, 4, one, 19, one, one, 1 << 30,
+                                 None, None) == B.ERR_BAD_ARG
+    assert L.specpc_token_select_static(ctypes.byref(pr), one, 1, 2, 7, 16, 8, 4, one, 1024, one, None, None) == B.ERR_BAD_ARG
+    assert L.spec_score(ctypes.byref(pr), one, one, None, 0, 2, one, one, 1 << 30, None, None) == B.ERR_BAD_ARG
+    # prompt compression
+    assert L.spec_gather_tokens(ctypes.byref(pr), one, None, None, 16, one, one, None, 64, one, None, None) == B.ERR_BAD_ARG
+    assert L.spec_gather_tokens(ctypes.byref(pr), one, one, one, 16, one, one, None, 64, one, None, None) == B.ERR_BAD_ARG
+    assert L.spec_gather_tokens(ctypes.byref(pr), one, None, one, 0, one, one, None, 64, one, None, None) == B.ERR_BAD_ARG
+    assert L.spec_gather_tokens(ctypes.byref(pr), one, None, one, 16, one, odd, None, 64, one, None, None) == B.ERR_ALIGNMENT
 
 
 def test_missing_library_fails_loudly(B, monkeypatch):
