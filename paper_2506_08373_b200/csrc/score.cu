@@ -36,10 +36,14 @@ constexpr int kEpilogueWarpgroups = 4;
 constexpr int kEpilogueThreads = kEpilogueWarpgroups * 128;
 constexpr int kMmaWarpB = 2 + kEpilogueThreads / 32;    // second MMA-issuing warp, after the epilogue warps
 constexpr int kThreads = 64 + kEpilogueThreads + 32;
-#ifndef SPEC_POLY_PAIRS
-#define SPEC_POLY_PAIRS 5
+#ifndef SPEC_POLY_PAIRS_1
+#define SPEC_POLY_PAIRS_1 5
 #endif
-constexpr int kPolyPairs = SPEC_POLY_PAIRS;   // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes
+#ifndef SPEC_POLY_PAIRS_2
+#define SPEC_POLY_PAIRS_2 5
+#endif
+// of the 16 element pairs in a 32-element block, evaluated on the FMA pipes (pass 1, pass 2)
+constexpr int kPolyPairs1 = SPEC_POLY_PAIRS_1, kPolyPairs2 = SPEC_POLY_PAIRS_2;
 constexpr int kBufCols = 128;                 // TMEM columns of a pass-2 accumulator buffer (pass 1 uses two of 256)
 constexpr int kTileKeys = 128;
 constexpr int kMaxStages = 8;
@@ -261,11 +265,11 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
   return make_float2(__uint_as_float(__float_as_uint(q.x) + (__float_as_uint(xr.x) << 23)),
                      __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(xr.y) << 23)));
 }
-// Pair i (0..15) of a 32-element block: kPolyPairs of them, evenly spread, avoid the MUFU unit.
-__device__ __forceinline__ constexpr bool poly_pair(int i) {
-  return (i * kPolyPairs) / 16 != ((i + 1) * kPolyPairs) / 16;
+// Pair i (0..15) of a 32-element block: NP of them, evenly spread, avoid the MUFU unit.
+template <int NP>
+__device__ __forceinline__ float2 ex2_pair(float2 x, int i) {
+  return (i * NP) / 16 != ((i + 1) * NP) / 16 ? ex2_poly2(x) : ex2_mufu2(x);
 }
-__device__ __forceinline__ float2 ex2_pair(float2 x, int i) { return poly_pair(i) ? ex2_poly2(x) : ex2_mufu2(x); }
 
 // Pass 1: fold 32 logits of one row into the running (max, sum-exp), log2 domain.  At least one
 // of the 32 logits is valid.
@@ -290,8 +294,8 @@ __device__ __forceinline__ void stats_update(const uint32_t (&r)[32], int valid,
   float2 s0 = splat2(0.f), s1 = splat2(0.f);
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
-    s0 = __fadd2_rn(s0, ex2_pair(__ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), a2, neg2), i));
-    s1 = __fadd2_rn(s1, ex2_pair(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1));
+    s0 = __fadd2_rn(s0, ex2_pair<kPolyPairs1>(__ffma2_rn(make_float2(v[2 * i], v[2 * i + 1]), a2, neg2), i));
+    s1 = __fadd2_rn(s1, ex2_pair<kPolyPairs1>(__ffma2_rn(make_float2(v[2 * i + 2], v[2 * i + 3]), a2, neg2), i + 1));
   }
   z += (s0.x + s0.y) + (s1.x + s1.y);
 }
@@ -304,8 +308,8 @@ __device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const f
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const float4 c = c4[i];
-    const float2 p0 = ex2_pair(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1])), a2, make_float2(c.x, c.y)), 2 * i);
-    const float2 p1 = ex2_pair(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), a2, make_float2(c.z, c.w)), 2 * i + 1);
+    const float2 p0 = ex2_pair<kPolyPairs2>(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1])), a2, make_float2(c.x, c.y)), 2 * i);
+    const float2 p1 = ex2_pair<kPolyPairs2>(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), a2, make_float2(c.z, c.w)), 2 * i + 1);
     if (MAXRED) {
       acc[0] = make_float2(fmaxf(acc[0].x, p0.x), fmaxf(acc[0].y, p0.y));
       acc[1] = make_float2(fmaxf(acc[1].x, p1.x), fmaxf(acc[1].y, p1.y));
