@@ -337,7 +337,7 @@ __device__ __forceinline__ bool locate_bin(const uint32_t* my_bins, int bins_per
 
 // Shared memory: top histogram, candidate keys and positions, candidate-pass histogram, a few
 // words of bookkeeping, then the parked groups (values and first positions) of all warps.
-constexpr int kTopkPendOffset = (kTopHistWords * 4 + 2 * kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2 + 1) * 4 + 15) / 16 * 16;
+constexpr int kTopkPendOffset = (kTopHistWords * 4 + 2 * kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2 + 2) * 4 + 15) / 16 * 16;
 constexpr int kTopkSmemBytes = kTopkPendOffset + kSelWarps * 32 * (kPerThread + 1) * 4;
 
 __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p) {
@@ -350,6 +350,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   int* out2 = wsum + kSelWarps;
   int* wcnt = out2 + 2;                                                  // [kSelWarps] list lengths, then the overflow flag
   int* overflow = wcnt + kSelWarps;
+  uint32_t* floor_pub = reinterpret_cast<uint32_t*>(overflow + 1);       // the highest floor any warp has located
   float* pend = reinterpret_cast<float*>(smem_raw + kTopkPendOffset);    // parked groups of all warps
 
   const int unit = blockIdx.x;
@@ -367,7 +368,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   if (take > 0 && take < e) {
     const SweepGeom g = make_geom(src, e, p.pool, p.pool_k);
     for (int i = tid; i < kTopHistWords; i += kSelThreads) top_hist[i] = 0;
-    if (tid == 0) *overflow = 0;
+    if (tid == 0) { *overflow = 0; *floor_pub = 0; }
     __syncthreads();
     uint32_t* ck = cand_key + warp * kWarpCap;
     int32_t* ci = cand_idx + warp * kWarpCap;
@@ -503,12 +504,22 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
         n_pend += n_hot;
         __syncwarp();
       }
-      if (((st + 1) & st) == 0 || (st & 31) == 31) expand();  // the histogram must be complete for the floor
-      if (((st + 1) & st) == 0 || (st & 31) == 31) {       // after steps 0, 1, 3, 7, 15, 31, then every 32nd
+      // The floor is kept fresh without stopping anybody: the warps take turns, one per step,
+      // to locate it on whatever the shared histogram holds (keys still parked, or a warp that
+      // lags, only make it lower, never wrong) and publish it; everybody picks it up each step.
+      if (st < 2) {
+        // the first two steps end with a CTA-wide update: every key so far is counted
+        expand();
         int fb, ab;
         if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, fb, ab))
           floor_key = max(floor_key, (uint32_t)fb << (32 - kTopBits));
+      } else if (warp == (st & (kSelWarps - 1))) {
+        const uint32_t before = floor_key;
+        warp_refloor();
+        if (floor_key != before && lane == 0) atomicMax(floor_pub, floor_key);
       }
+      const uint32_t pub = *reinterpret_cast<volatile uint32_t*>(floor_pub);
+      if (pub > floor_key) floor_key = pub;
     };
 
     if (max7) {
