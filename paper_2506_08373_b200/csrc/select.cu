@@ -301,6 +301,14 @@ __device__ __forceinline__ void pool_max7(const float4 (&w4)[4], float (&val)[kP
 // with 16-byte loads, and the padding staggers the lanes over the memory banks.
 __device__ __forceinline__ int top_word(uint32_t b) { return (int)(b + ((b >> 8) << 2)); }
 
+// Bin of a key in the top-bits histogram.  Scores are sums or maxima of probabilities, so their
+// keys have the sign bit set: the bins spend all kTopBits bits on exponent and mantissa (bits
+// 30..18, 3 % wide) and every negative score falls into bin 0.  A threshold inside bin 0 (a
+// negative or vanishing score) takes the generic path.
+constexpr int kTopShift = 31 - kTopBits;
+__device__ __forceinline__ uint32_t top_bin(uint32_t key) { return key & 0x80000000u ? (key & 0x7fffffffu) >> kTopShift : 0u; }
+__device__ __forceinline__ uint32_t bin_floor_key(uint32_t bin) { return bin ? 0x80000000u | (bin << kTopShift) : 0u; }
+
 // Finds the bin holding the need-th largest element of a histogram whose bins are spread
 // over the threads, bins_per_thread consecutive bins each starting at my_bins (need >= 1).  Returns the bin and
 // the number of elements in higher bins to every thread; false (outputs untouched) when the
@@ -411,7 +419,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       }
       const uint32_t who = __ballot_sync(0xffffffffu, here);
       if (who) {
-        const uint32_t fk = (uint32_t)__shfl_sync(0xffffffffu, bin, __ffs(who) - 1) << (32 - kTopBits);
+        const uint32_t fk = bin_floor_key((uint32_t)__shfl_sync(0xffffffffu, bin, __ffs(who) - 1));
         if (fk > floor_key) floor_key = fk;
       }
     };
@@ -466,7 +474,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       const int total = __shfl_sync(0xffffffffu, incl, 31);
 #pragma unroll
       for (int u = 0; u < kPerThread; ++u)
-        if (take_mask & (1u << u)) atomicAdd(&top_hist[top_word(to_key(val[u]) >> (32 - kTopBits))], 1u);
+        if (take_mask & (1u << u)) atomicAdd(&top_hist[top_word(top_bin(to_key(val[u])))], 1u);
       if (cnt + total > kWarpCap) filter_list();
       if (cnt + total > kWarpCap) { warp_refloor(); filter_list(); }   // my list alone is too long: fresher floor
       if (cnt + total <= kWarpCap) {
@@ -512,7 +520,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
         expand();
         int fb, ab;
         if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, fb, ab))
-          floor_key = max(floor_key, (uint32_t)fb << (32 - kTopBits));
+          floor_key = max(floor_key, bin_floor_key((uint32_t)fb));
       } else if (warp == (st & (kSelWarps - 1))) {
         const uint32_t before = floor_key;
         warp_refloor();
@@ -554,12 +562,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     if (lane == 0) wcnt[warp] = cnt;
     int b1 = 0, above = 0;
     bool fits = locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
-    fits = fits && *overflow == 0;
+    fits = fits && *overflow == 0 && b1 > 0;                 // bin 0 mixes keys with different leading bits
     if (fits) {
       // ---- remaining bits on the candidates only (every warp walks its own list)
-      int known = kTopBits;
-      uint32_t prefix = (uint32_t)b1 << (32 - kTopBits);
-      uint32_t mask = ~((1u << (32 - kTopBits)) - 1u);
+      int known = kTopBits + 1;                              // the sign bit and the bin
+      uint32_t prefix = bin_floor_key((uint32_t)b1);
+      uint32_t mask = ~((1u << kTopShift) - 1u);
       int remaining = take - above;
       while (known < 32) {
         const int w = min(10, 32 - known), shift = 32 - known - w;
