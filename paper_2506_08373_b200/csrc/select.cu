@@ -301,14 +301,6 @@ __device__ __forceinline__ void pool_max7(const float4 (&w4)[4], float (&val)[kP
 // with 16-byte loads, and the padding staggers the lanes over the memory banks.
 __device__ __forceinline__ int top_word(uint32_t b) { return (int)(b + ((b >> 8) << 2)); }
 
-// Bin of a key in the top-bits histogram.  Scores are sums or maxima of probabilities, so their
-// keys have the sign bit set: the bins spend all kTopBits bits on exponent and mantissa (bits
-// 30..18, 3 % wide) and every negative score falls into bin 0.  A threshold inside bin 0 (a
-// negative or vanishing score) takes the generic path.
-constexpr int kTopShift = 31 - kTopBits;
-__device__ __forceinline__ uint32_t top_bin(uint32_t key) { return key & 0x80000000u ? (key & 0x7fffffffu) >> kTopShift : 0u; }
-__device__ __forceinline__ uint32_t bin_floor_key(uint32_t bin) { return bin ? 0x80000000u | (bin << kTopShift) : 0u; }
-
 // Finds the bin holding the need-th largest element of a histogram whose bins are spread
 // over the threads, bins_per_thread consecutive bins each starting at my_bins (need >= 1).  Returns the bin and
 // the number of elements in higher bins to every thread; false (outputs untouched) when the
@@ -345,7 +337,7 @@ __device__ __forceinline__ bool locate_bin(const uint32_t* my_bins, int bins_per
 
 // Shared memory: top histogram, candidate keys and positions, candidate-pass histogram, a few
 // words of bookkeeping, then the parked groups (values and first positions) of all warps.
-constexpr int kTopkPendOffset = (kTopHistWords * 4 + 2 * kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2 + 2) * 4 + 15) / 16 * 16;
+constexpr int kTopkPendOffset = (kTopHistWords * 4 + 2 * kCandCap * 4 + kFinBins * 4 + (2 * kSelWarps + 2 + 1) * 4 + 15) / 16 * 16;
 constexpr int kTopkSmemBytes = kTopkPendOffset + kSelWarps * 32 * (kPerThread + 1) * 4;
 
 __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p) {
@@ -358,7 +350,6 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   int* out2 = wsum + kSelWarps;
   int* wcnt = out2 + 2;                                                  // [kSelWarps] list lengths, then the overflow flag
   int* overflow = wcnt + kSelWarps;
-  uint32_t* floor_pub = reinterpret_cast<uint32_t*>(overflow + 1);       // the highest floor any warp has located
   float* pend = reinterpret_cast<float*>(smem_raw + kTopkPendOffset);    // parked groups of all warps
 
   const int unit = blockIdx.x;
@@ -376,7 +367,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
   if (take > 0 && take < e) {
     const SweepGeom g = make_geom(src, e, p.pool, p.pool_k);
     for (int i = tid; i < kTopHistWords; i += kSelThreads) top_hist[i] = 0;
-    if (tid == 0) { *overflow = 0; *floor_pub = 0; }
+    if (tid == 0) *overflow = 0;
     __syncthreads();
     uint32_t* ck = cand_key + warp * kWarpCap;
     int32_t* ci = cand_idx + warp * kWarpCap;
@@ -419,7 +410,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       }
       const uint32_t who = __ballot_sync(0xffffffffu, here);
       if (who) {
-        const uint32_t fk = bin_floor_key((uint32_t)__shfl_sync(0xffffffffu, bin, __ffs(who) - 1));
+        const uint32_t fk = (uint32_t)__shfl_sync(0xffffffffu, bin, __ffs(who) - 1) << (32 - kTopBits);
         if (fk > floor_key) floor_key = fk;
       }
     };
@@ -474,7 +465,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
       const int total = __shfl_sync(0xffffffffu, incl, 31);
 #pragma unroll
       for (int u = 0; u < kPerThread; ++u)
-        if (take_mask & (1u << u)) atomicAdd(&top_hist[top_word(top_bin(to_key(val[u])))], 1u);
+        if (take_mask & (1u << u)) atomicAdd(&top_hist[top_word(to_key(val[u]) >> (32 - kTopBits))], 1u);
       if (cnt + total > kWarpCap) filter_list();
       if (cnt + total > kWarpCap) { warp_refloor(); filter_list(); }   // my list alone is too long: fresher floor
       if (cnt + total <= kWarpCap) {
@@ -512,22 +503,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
         n_pend += n_hot;
         __syncwarp();
       }
-      // The floor is kept fresh without stopping anybody: the warps take turns, one per step,
-      // to locate it on whatever the shared histogram holds (keys still parked, or a warp that
-      // lags, only make it lower, never wrong) and publish it; everybody picks it up each step.
-      if (st < 2) {
-        // the first two steps end with a CTA-wide update: every key so far is counted
-        expand();
+      if (((st + 1) & st) == 0 || (st & 31) == 31) expand();  // the histogram must be complete for the floor
+      if (((st + 1) & st) == 0 || (st & 31) == 31) {       // after steps 0, 1, 3, 7, 15, 31, then every 32nd
         int fb, ab;
         if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, fb, ab))
-          floor_key = max(floor_key, bin_floor_key((uint32_t)fb));
-      } else if (warp == (st & (kSelWarps - 1))) {
-        const uint32_t before = floor_key;
-        warp_refloor();
-        if (floor_key != before && lane == 0) atomicMax(floor_pub, floor_key);
+          floor_key = max(floor_key, (uint32_t)fb << (32 - kTopBits));
       }
-      const uint32_t pub = *reinterpret_cast<volatile uint32_t*>(floor_pub);
-      if (pub > floor_key) floor_key = pub;
     };
 
     if (max7) {
@@ -562,12 +543,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     if (lane == 0) wcnt[warp] = cnt;
     int b1 = 0, above = 0;
     bool fits = locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
-    fits = fits && *overflow == 0 && b1 > 0;                 // bin 0 mixes keys with different leading bits
+    fits = fits && *overflow == 0;
     if (fits) {
       // ---- remaining bits on the candidates only (every warp walks its own list)
-      int known = kTopBits + 1;                              // the sign bit and the bin
-      uint32_t prefix = bin_floor_key((uint32_t)b1);
-      uint32_t mask = ~((1u << kTopShift) - 1u);
+      int known = kTopBits;
+      uint32_t prefix = (uint32_t)b1 << (32 - kTopBits);
+      uint32_t mask = ~((1u << (32 - kTopBits)) - 1u);
       int remaining = take - above;
       while (known < 32) {
         const int w = min(10, 32 - known), shift = 32 - known - w;
