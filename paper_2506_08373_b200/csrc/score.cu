@@ -84,6 +84,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One arrival for the whole warp, after a warp-wide (.sync.aligned) instruction has completed
+// for all lanes: predicated, no branch.
+__device__ __forceinline__ void arrive_lane0(uint64_t* bar, int lane) {
+  asm volatile("{\n.reg .pred p;\nsetp.eq.s32 p, %1, 0;\n@p mbarrier.arrive.shared::cta.b64 _, [%0];\n}"
+               ::"r"(smem_u32(bar)), "r"(lane) : "memory");
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -92,7 +98,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait.  Returns false when another role has given up or the time limit passed.  The
 // suspend-time hint lets the hardware park the thread until the phase completes instead of
 // spinning in the issue slots the epilogue warps need.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const uint32_t addr = smem_u32(bar);
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -548,34 +554,38 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           const int n_item = t + 1 < sg.nt ? 2 * kTileKeys : kTileKeys;            // the last item of an odd segment is one tile
           const int key0 = (sg.t0 + t) * kTileKeys;                                // first key of the item
           const int nvh = min(n_item, sg.n - key0) - wg * 64;                      // valid keys in my 64 columns
+          const bool in_window = p.causal && key0 + n_item > sg.n - p.n_window;    // warp-uniform
+          const bool plain = nvh >= 64 && !in_window;
           for (int mt = 0; mt < n_mt; ++mt, ++bit) {
             const int buf = (int)(bit & 1u);
             ok = mbar_wait(&t_full[buf], (bit >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             float m = mrun[mt], z = zrun[mt];
-            int vis2 = 0;                                    // visible keys of the second 32 columns
-            if (nvh > 0) {
-              const uint32_t taddr = lane_base + buf * 256 + wg * 64;
-              // keys of my 64 columns that this thread's row may see
-              int vis = nvh;
-              const bool in_window = p.causal && key0 + n_item > sg.n - p.n_window;   // warp-uniform
-              if (in_window) {
-                const int rr = (mt * 128 + row_in_tile) % p.R;
-                if (rr < p.n_window) vis = min(nvh, max(sg.n - p.n_window + rr, 0) + 1 - (key0 + wg * 64));
-              }
+            const uint32_t taddr = lane_base + buf * 256 + wg * 64;
+            if (plain) {
+              // all 64 of my columns are keys every row sees: no masks, no per-row arithmetic
               tmem_ld32(taddr, ra);
-              if (!in_window && nvh >= 32) stats_update<false>(ra, 32, p.a, m, z);
-              else if (vis > 0) stats_update<true>(ra, min(vis, 32), p.a, m, z);
-              if (nvh > 32) tmem_ld32(taddr + 32, ra);
-              vis2 = in_window || nvh < 64 ? vis - 32 : 32;
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&t_empty[buf]);       // all reads done: the buffer can be refilled
-            if (nvh > 32) {
-              if (vis2 >= 32 && nvh >= 64) stats_update<false>(ra, 32, p.a, m, z);
-              else if (vis2 > 0) stats_update<true>(ra, min(vis2, 32), p.a, m, z);
+              stats_update<false>(ra, 32, p.a, m, z);
+              tmem_ld32(taddr + 32, ra);
+              tc_fence_before();
+              arrive_lane0(&t_empty[buf], lane);               // all reads done: the buffer can be refilled
+              stats_update<false>(ra, 32, p.a, m, z);
+            } else {
+              int vis = nvh, vis2 = 0;                         // keys of my 64 columns that this thread's row may see
+              if (nvh > 0) {
+                if (in_window) {
+                  const int rr = (mt * 128 + row_in_tile) % p.R;
+                  if (rr < p.n_window) vis = min(nvh, max(sg.n - p.n_window + rr, 0) + 1 - (key0 + wg * 64));
+                }
+                tmem_ld32(taddr, ra);
+                if (vis > 0) stats_update<true>(ra, min(vis, 32), p.a, m, z);
+                if (nvh > 32) tmem_ld32(taddr + 32, ra);
+                vis2 = vis - 32;
+              }
+              tc_fence_before();
+              arrive_lane0(&t_empty[buf], lane);
+              if (nvh > 32 && vis2 > 0) stats_update<true>(ra, min(vis2, 32), p.a, m, z);
             }
             mrun[mt] = m;
             zrun[mt] = z;
@@ -625,8 +635,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
               tmem_ld32(taddr + 32, ra);
             }
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&t_empty[buf]);
+            arrive_lane0(&t_empty[buf], lane);
             if (!in_window) prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
             else prob_accumulate_causal<MAXRED>(ra, hw > 32 ? negc + 32 : negc, p.a, acc, hw > 32 ? row0 + 32 : row0, p.R, p.n_window, sg.n, key);
           }
