@@ -114,7 +114,11 @@ const char* spec_last_error(void);
  *              its own prompt position n_s - n_window + r.
  *  scores_out  [n_layers, n_kv_heads, T] fp32; the whole buffer is overwritten (tokens that no
  *              sequence covers are set to 0)
- * Limits: M*head_dim <= 81920 (e.g. M <= 640 at head_dim 128); else SPEC_ERR_UNSUPPORTED.
+ * Query rows: up to M*head_dim = 81920 (M <= 640 at head_dim 128, 1280 at 64) are scored in one
+ * sweep over the keys and the result is bit-reproducible from run to run; a larger M (a long
+ * lookahead, a wide GQA group) is scored in ceil(M / that many) sweeps over equal groups of rows,
+ * whose contributions are added in scores_out (SUM then rounds in an order that may differ between
+ * runs, within the fp32 tolerance).
  */
 int32_t spec_score(const spec_problem* problem, const void* q, const void* k, const float* row_weight,
                    int32_t reduce, int32_t causal_window, float* scores_out, void* workspace,

@@ -29,6 +29,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include <algorithm>
 
 namespace spec {
 
@@ -63,7 +64,8 @@ struct ScoreParams {
   float* scores;        // [L, Hkv, T]
   int32_t* status;
   long long T;
-  int n_in, n_seq, L, Hq, Hkv, G, R, M, M_pad, d;
+  int n_in, n_seq, L, Hq, Hkv, G, R, M, M_pad, d;   // M, M_pad: the query rows of this launch, rows [row0, row0 + M) of every unit
+  int row0;
   int causal, n_window;  // causal != 0: window row r sees keys up to position n - n_window + r only
   int n_stages, n_chunks, cw_last;   // pass 2: chunks of 128 query rows, the last of cw_last (64 or 128)
   int reduce;
@@ -414,7 +416,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
         for (int kh = 0; kh < n_kh; ++kh)
           for (int rb = 0; rb < p.M_pad / 128; ++rb)
-            tma_load_2d(q_sm + kh * q_half_bytes + rb * (128 * 128), &tm_q, kh * 64, qrow0 + rb * 128, q_full);
+            tma_load_2d(q_sm + kh * q_half_bytes + rb * (128 * 128), &tm_q, kh * 64, qrow0 + p.row0 + rb * 128, q_full);
         for (int t = 0; t < sg.nt; ++t, ++kit) {
           const int stage = kit % p.n_stages;
           const uint32_t par = (kit / p.n_stages) & 1;
@@ -575,7 +577,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
               int vis = nvh, vis2 = 0;                         // keys of my 64 columns that this thread's row may see
               if (nvh > 0) {
                 if (in_window) {
-                  const int rr = (mt * 128 + row_in_tile) % p.R;
+                  const int rr = (p.row0 + mt * 128 + row_in_tile) % p.R;
                   if (rr < p.n_window) vis = min(nvh, max(sg.n - p.n_window + rr, 0) + 1 - (key0 + wg * 64));
                 }
                 tmem_ld32(taddr, ra);
@@ -612,7 +614,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
       while (seg_next(it, p, tp, sg)) {
         const int qrow0 = ((sg.s * p.L + sg.l) * p.Hq + sg.h * p.G) * p.R;
         asm volatile("bar.sync 1, 512;" ::: "memory");          // previous unit's constants no longer read
-        for (int i = et; i < p.M_pad; i += kEpilogueThreads) c_sm[i] = i < p.M ? p.rowc[qrow0 + i] : -INFINITY;
+        for (int i = et; i < p.M_pad; i += kEpilogueThreads) c_sm[i] = i < p.M ? p.rowc[qrow0 + p.row0 + i] : -INFINITY;
         asm volatile("bar.sync 1, 512;" ::: "memory");
         float* out = p.scores + ((long long)sg.l * p.Hkv + sg.h) * p.T + sg.begin;
         for (int t = pair; t < sg.nt && ok; t += 2) {
@@ -627,7 +629,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const int hw = (ch == p.n_chunks - 1 ? p.cw_last : 128) >> 1;     // my columns: 32 or 64
             const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
             const float* negc = c_sm + ch * 128 + half * hw;
-            const int row0 = ch * 128 + half * hw;              // query row of my first column
+            const int row0 = p.row0 + ch * 128 + half * hw;     // query row of my first column
             tmem_ld32(taddr, ra);
             if (hw > 32) {
               if (!in_window) prob_accumulate<MAXRED>(ra, negc, a2, acc);
@@ -709,8 +711,8 @@ __global__ void __launch_bounds__(128) merge_kernel(const ScoreParams p, int n_c
       if (pm > -INFINITY) z += pz * exp2f(pm - m);
     }
     float c = m + log2f(z);
-    if (p.row_weight) c -= log2f(p.row_weight[i % p.R]);
-    p.rowc[qrow0 + i] = -c;
+    if (p.row_weight) c -= log2f(p.row_weight[(p.row0 + i) % p.R]);
+    p.rowc[qrow0 + p.row0 + i] = -c;
   }
 }
 
@@ -752,9 +754,11 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   const int R = pr->n_lookahead + pr->n_window;
   const int G = pr->n_q_heads / pr->n_kv_heads;
   const int M = G * R;
-  const int M_pad = (M + 127) / 128 * 128;
-  if ((int64_t)M_pad * d > 81920 || M_pad / 128 > kMaxMTiles)
-    return fail(SPEC_ERR_UNSUPPORTED, "G*R=%d query rows per KV head at head_dim=%d exceed the resident-query limit (G*R*head_dim <= 81920)", M, d);
+  // The query rows of a unit stay resident in shared memory; more than fit (G*R*head_dim > 81920) are
+  // scored in several launches over equal groups of rows, whose contributions add up in scores_out.
+  const int rows_max = std::min(81920 / d, kMaxMTiles * 128) / 128 * 128;
+  const int n_groups = (M + rows_max - 1) / rows_max;
+  const int rows_group = ((M + n_groups - 1) / n_groups + 127) / 128 * 128;
   const WorkspacePlan wp = plan_workspace(pr);
   if (!workspace || workspace_bytes < wp.total)
     return fail(SPEC_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", workspace_bytes, wp.total);
@@ -798,39 +802,48 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   p.status = status_word;
   p.T = pr->total_tokens;
   p.n_in = pr->n_in; p.n_seq = pr->n_seq; p.L = pr->n_layers; p.Hq = pr->n_q_heads; p.Hkv = pr->n_kv_heads;
-  p.G = G; p.R = R; p.M = M; p.M_pad = M_pad; p.d = d;
-  const int M64 = (M + 63) / 64 * 64;                      // pass 2 splits each chunk's columns in two halves of 32 or 64
-  p.n_chunks = (M64 + 127) / 128;
-  p.cw_last = M64 - (p.n_chunks - 1) * 128;
+  p.G = G; p.R = R; p.d = d;
   p.reduce = reduce;
   p.causal = causal_window;
   p.n_window = pr->n_window;
   p.a = (float)((double)pr->softmax_scale * 1.4426950408889634);
-  p.q_bytes = (uint32_t)M_pad * d * 2;
   p.stage_bytes = (uint32_t)kTileKeys * d * 2;
-  const int small = M_pad * 4 + (pr->n_seq + 1) * 4 + 8 + kNumBars * 8 + 16;
-  const int smem_max = 227 * 1024;
-  int stages = (smem_max - (int)p.q_bytes - small) / (int)p.stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  stages &= ~1;                                            // pass 1 consumes the ring two stages at a time
-  if (stages < 2) return fail(SPEC_ERR_UNSUPPORTED, "not enough shared memory for two key stages (M=%d, head_dim=%d)", M, d);
-  p.n_stages = stages;
-  int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
-  if (smem < 120 * 1024) smem = 120 * 1024;               // one CTA per SM: each CTA owns the whole TMEM
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int n_ctas = wp.score_ctas;
   const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
   auto pass1 = score_kernel<1, false>;
   auto pass2 = reduce == SPEC_REDUCE_MAX ? score_kernel<2, true> : score_kernel<2, false>;
-  SPEC_CUDA_OK(cudaFuncSetAttribute(pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  SPEC_CUDA_OK(cudaFuncSetAttribute(pass2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   SPEC_CUDA_OK(cudaMemsetAsync(scores_out, 0, (size_t)pr->n_layers * pr->n_kv_heads * (size_t)pr->total_tokens * sizeof(float), st));
-  pass1<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
-  SPEC_CUDA_OK(cudaGetLastError());
-  merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);
-  SPEC_CUDA_OK(cudaGetLastError());
-  pass2<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
-  SPEC_CUDA_OK(cudaGetLastError());
+  int smem_set = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    p.row0 = g * rows_group;
+    p.M = std::min(rows_group, M - p.row0);
+    p.M_pad = (p.M + 127) / 128 * 128;
+    const int M64 = (p.M + 63) / 64 * 64;                  // pass 2 splits each chunk's columns in two halves of 32 or 64
+    p.n_chunks = (M64 + 127) / 128;
+    p.cw_last = M64 - (p.n_chunks - 1) * 128;
+    p.q_bytes = (uint32_t)p.M_pad * d * 2;
+    const int small = p.M_pad * 4 + (pr->n_seq + 1) * 4 + 8 + kNumBars * 8 + 16;
+    const int smem_max = 227 * 1024;
+    int stages = (smem_max - (int)p.q_bytes - small) / (int)p.stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    stages &= ~1;                                          // pass 1 consumes the ring two stages at a time
+    if (stages < 2) return fail(SPEC_ERR_UNSUPPORTED, "not enough shared memory for two key stages (%d rows, head_dim=%d)", p.M, d);
+    p.n_stages = stages;
+    int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
+    if (smem < 120 * 1024) smem = 120 * 1024;             // one CTA per SM: each CTA owns the whole TMEM
+    if (smem > smem_set) {
+      SPEC_CUDA_OK(cudaFuncSetAttribute(pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      SPEC_CUDA_OK(cudaFuncSetAttribute(pass2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      smem_set = smem;
+    }
+    pass1<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+    SPEC_CUDA_OK(cudaGetLastError());
+    merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);
+    SPEC_CUDA_OK(cudaGetLastError());
+    pass2<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
+    SPEC_CUDA_OK(cudaGetLastError());
+  }
   return SPEC_OK;
 }

@@ -38,6 +38,10 @@ SCORE_CASES = {
     "d64_M5_one_head": lambda W: (small(W, head_dim=64, n_q_heads=2, n_kv_heads=2, n_lookahead=3, n_window=2,
                                         zipf_bias=False, n_in=777), [0]),
     "d128_M21": lambda W: (small(W, n_q_heads=6, n_kv_heads=2, n_lookahead=4, n_window=3, n_in=300), [0, 1]),
+    # more query rows than stay resident in shared memory: scored in several groups of rows
+    "d128_M800_two_row_groups": lambda W: (small(W, n_lookahead=168, n_in=1500), [0]),
+    "d128_G8_M1536_three_row_groups": lambda W: (small(W, n_q_heads=16, n_kv_heads=2, n_lookahead=160, n_in=700), [0, 1]),
+    "d64_M1400_two_row_groups": lambda W: (small(W, head_dim=64, n_lookahead=318, n_in=900), [0]),
     "snapkv_no_lookahead": lambda W: (small(W, n_lookahead=0, n_in=513), [0]),
     "single_key": lambda W: (small(W, n_in=1, zipf_bias=False, planted="singletons", n_planted=0), [0]),
     "ragged_batch": lambda W: (W.CONFIGS[4].replace(n_layers=2, n_seq=7, len_lo=1, len_hi=900, c_max=64), [0, 1]),
@@ -100,6 +104,15 @@ def test_score_max_reduce_and_row_weights(B, W, oracle):
     ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale, mode=oracle.MAX)
     assert_scores_close(got, ref, g.cu)
     assert got.max() <= 1.0 + 1e-5
+    # the same over several groups of rows (G * R = 840 > 640): weights and the causal window follow the row index
+    w = small(W, n_in=700, n_lookahead=170, n_window=40)
+    g = Gpu(B, W, w, [0])
+    rw = torch.linspace(1.0 / w.rows, 1.0, w.rows)
+    for reduce in (B.REDUCE_SUM, B.REDUCE_MAX):
+        got = g.score(reduce=reduce, row_weight=rw.cuda(), causal_window=1).cpu().numpy()
+        ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale,
+                                row_weight=rw.double().numpy(), mode=reduce, causal_window=True)
+        assert_scores_close(got, ref, g.cu)
 
 
 def test_score_causal_window(B, W, oracle):
@@ -137,12 +150,13 @@ def test_score_token_major_key_layout_and_reproducibility(B, W, oracle):
     assert torch.equal(g.score(), base)
 
 
-def test_score_rejects_unsupported_shapes(B, W):
-    w = small(W, n_q_heads=64, n_kv_heads=2)               # 32*96 rows per KV head
+def test_score_wide_gqa_group_in_five_row_groups(B, W, oracle):
+    w = small(W, n_q_heads=64, n_kv_heads=2, n_in=400)     # 32 * 96 = 3072 query rows per KV head
     g = Gpu(B, W, w, [0])
-    with pytest.raises(B.SpecError) as e:
-        g.score()
-    assert e.value.code == B.ERR_UNSUPPORTED
+    got = g.score().cpu().numpy()
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale)
+    assert_scores_close(got, ref, g.cu)
+    np.testing.assert_allclose(got.astype(np.float64).sum(-1), w.group * w.rows, rtol=1e-4)
 
 
 # ------------------------------------------------------------------ selection ---------

@@ -68,8 +68,6 @@ def test_bad_call_arguments_are_rejected_on_the_host(B):
     assert L.spec_score(ctypes.byref(pr), odd, one, None, 0, 0, one, one, 1 << 30, None, None) == B.ERR_ALIGNMENT
     assert L.spec_score(ctypes.byref(pr), one, one, None, 5, 0, one, one, 1 << 30, None, None) == B.ERR_BAD_ARG
     assert L.spec_score(ctypes.byref(pr), one, one, None, 0, 0, one, one, 8, None, None) == B.ERR_WORKSPACE
-    big = good_problem(B, n_q_heads=64, n_kv_heads=2, n_lookahead=64, n_window=32, head_dim=128)
-    assert L.spec_score(ctypes.byref(big), one, one, None, 0, 0, one, one, 1 << 40, None, None) == B.ERR_UNSUPPORTED
     assert L.spec_pool_topk(ctypes.byref(pr), one, 0, 0, 16, 0, one, None, None, 0, None, None) == B.ERR_BAD_ARG
     assert L.spec_pool_topk(ctypes.byref(pr), one, 0, 7, 16, 17, one, None, None, 0, None, None) == B.ERR_BAD_ARG
     assert L.spec_pool_topk(ctypes.byref(pr), one, 3, 7, 16, 0, one, None, None, 0, None, None) == B.ERR_BAD_ARG
