@@ -319,8 +319,8 @@ __device__ __forceinline__ void prob_accumulate(const uint32_t (&r)[32], const f
     const float2 p0 = ex2_pair<kPolyPairs2>(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1])), a2, make_float2(c.x, c.y)), 2 * i);
     const float2 p1 = ex2_pair<kPolyPairs2>(__ffma2_rn(make_float2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), a2, make_float2(c.z, c.w)), 2 * i + 1);
     if (MAXRED) {
-      acc[0] = make_float2(fmaxf(acc[0].x, p0.x), fmaxf(acc[0].y, p0.y));
-      acc[1] = make_float2(fmaxf(acc[1].x, p1.x), fmaxf(acc[1].y, p1.y));
+      acc[0].x = max3(acc[0].x, p0.x, p0.y);               // one maximum per chain: the four are merged at the end
+      acc[1].x = max3(acc[1].x, p1.x, p1.y);
     } else {
       acc[0] = __fadd2_rn(acc[0], p0);
       acc[1] = __fadd2_rn(acc[1], p1);
