@@ -7,8 +7,11 @@
  * built on the same scores (Algorithm 2, lines 7-10).
  *
  * Conventions for every entry point
- *   - All data pointers are DEVICE pointers owned by the caller.  The library
- *     never allocates, frees or retains them.  Scratch memory is passed in as
+ *   - All data pointers are DEVICE pointers owned by the caller (any memory the
+ *     device can address: device memory, or page-locked host memory mapped into
+ *     the device's address space, which suits a source that is read sparsely,
+ *     such as v in spec_compact_kv).  The library never allocates, frees or
+ *     retains them.  Scratch memory is passed in as
  *     `workspace` (size from spec_workspace_bytes); its contents are undefined
  *     on entry and on return.
  *   - Work is enqueued asynchronously on `stream` (a cudaStream_t passed as

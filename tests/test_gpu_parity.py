@@ -269,6 +269,13 @@ def test_compact_bit_exact_contiguous_and_paged(B, W, oracle, d):
     assert status.item() == 0
     np.testing.assert_array_equal(bits(ko), oracle.compact(bits(k), cu, idx))
     np.testing.assert_array_equal(bits(vo), oracle.compact(bits(v), cu, idx))
+    # V left in page-locked host memory: only the selected rows cross the bus
+    v_host = v.cpu().pin_memory()
+    vo.fill_(1.0)
+    B.spec_compact_kv(pr, k, v_host, idx_t, C, ko, vo, status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    np.testing.assert_array_equal(bits(vo), oracle.compact(bits(v), cu, idx))
     # K only
     ko.fill_(1.0)
     B.spec_compact_kv(pr, k, None, idx_t, C, ko, None, status_word=status)
