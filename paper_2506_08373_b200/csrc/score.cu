@@ -38,10 +38,10 @@ constexpr int kEpilogueThreads = kEpilogueWarpgroups * 128;
 constexpr int kMmaWarpB = 2 + kEpilogueThreads / 32;    // second MMA-issuing warp, after the epilogue warps
 constexpr int kThreads = 64 + kEpilogueThreads + 32;
 #ifndef SPEC_POLY_PAIRS_1
-#define SPEC_POLY_PAIRS_1 5
+#define SPEC_POLY_PAIRS_1 4
 #endif
 #ifndef SPEC_POLY_PAIRS_2
-#define SPEC_POLY_PAIRS_2 5
+#define SPEC_POLY_PAIRS_2 4
 #endif
 // of the 16 element pairs in a 32-element block, evaluated on the FMA pipes (pass 1, pass 2)
 constexpr int kPolyPairs1 = SPEC_POLY_PAIRS_1, kPolyPairs2 = SPEC_POLY_PAIRS_2;
