@@ -19,7 +19,7 @@ constexpr int kSmemLimit = 227 * 1024;
 
 // Monotone map float -> uint32 (larger float <=> larger key), valid for any sign.
 __device__ __forceinline__ uint32_t to_key(float v) {
-  const uint32_t b = __float_as_uint(v);
+  const uint32_t b = __float_as_uint(v + 0.0f);            // -0.0 + 0.0 = +0.0: the two zeros tie, as they compare equal
   return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);   // negative: all bits flipped; else: sign bit set
 }
 

@@ -231,6 +231,36 @@ def test_topk_clustered_keys_large_budget_and_odd_offsets(B, W, oracle):
     run_topk_case(B, W, oracle, scores, [0, 4099, 4099 + 33333, 4099 + 33333 + 12345], 0, 7, 512, 40)
 
 
+def test_topk_seeded_random_shapes_and_special_values(B, W, oracle):
+    """Many small seeded cases: lengths around tile and vector edges, budgets from 1 to beyond n, odd
+    pooling widths, forced tails, and score vectors with negatives, signed zeros, infinities and
+    long runs of equal values.  Max-pool selection is exact, ties to the lower position."""
+    rng = np.random.default_rng(2024)
+    for case in range(48):
+        n_seq = int(rng.integers(1, 4))
+        lens = [int(rng.choice([0, 1, 2, 7, 31, 127, 128, 129, 1000, int(rng.integers(1, 6000))])) for _ in range(n_seq)]
+        if sum(lens) == 0:
+            lens[0] = 5
+        cu = [0] + list(np.cumsum(lens))
+        T = cu[-1] + int(rng.integers(0, 5))                   # a few tokens no sequence covers
+        kind = case % 4
+        if kind == 0:
+            x = rng.standard_normal((2, 2, T)).astype(np.float32)
+        elif kind == 1:
+            x = (rng.integers(0, 4, size=(2, 2, T)) * 0.25).astype(np.float32)          # long runs of ties
+        elif kind == 2:
+            x = rng.random((2, 2, T)).astype(np.float32) ** 10
+            x[rng.random(x.shape) < 0.02] = np.inf
+            x[rng.random(x.shape) < 0.02] = -np.inf
+        else:
+            x = np.where(rng.random((2, 2, T)) < 0.5, np.float32(0.0), np.float32(-0.0)).astype(np.float32)
+            x[rng.random(x.shape) < 0.1] = 1e-30
+        k = int(rng.choice([1, 3, 5, 7, 9, 31]))
+        c_max = int(rng.choice([1, 2, 16, 100, 1024, max(lens) + 3]))
+        forced = int(rng.integers(0, min(c_max, 20) + 1)) if case % 3 == 0 else 0
+        run_topk_case(B, W, oracle, x, cu, 0, k, c_max, forced)
+
+
 def test_topk_avg_pool_within_band(B, W, oracle):
     rng = np.random.default_rng(3)
     scores = rng.random((1, 2, 3000)).astype(np.float32) ** 4
