@@ -135,6 +135,33 @@ def test_score_causal_window(B, W, oracle):
     assert torch.allclose(a.sum(-1), b.sum(-1), rtol=1e-4)              # rows still sum to one
 
 
+def test_score_seeded_random_geometry(B, W, oracle):
+    """Seeded sweep over GQA group sizes, row counts, head sizes, single and ragged batches, both
+    reductions, the causal window and row weights, each against the oracle."""
+    rng = np.random.default_rng(77)
+    for case in range(16):
+        hkv = int(rng.choice([1, 2]))
+        group = int(rng.choice([1, 2, 3, 4, 7]))
+        kw = dict(head_dim=int(rng.choice([64, 128])), n_kv_heads=hkv, n_q_heads=hkv * group,
+                  n_lookahead=int(rng.integers(0, 41)), n_window=int(rng.integers(1, 41)), seed=100 + case,
+                  zipf_bias=bool(case % 2), n_planted=4)
+        if case % 3 == 0:
+            w = W.CONFIGS[4].replace(n_layers=1, n_seq=int(rng.integers(2, 5)), len_lo=0, len_hi=int(rng.integers(1, 700)),
+                                     c_max=8, **kw)
+        else:
+            w = small(W, n_layers=1, n_in=int(rng.choice([1, 5, 127, 128, 129, 255, 257, 700, 1500])), **kw)
+        g = Gpu(B, W, w, [0])
+        reduce = int(case % 2)
+        causal = bool((case // 2) % 2)
+        rw = None
+        if case % 4 == 3:
+            rw = torch.from_numpy(rng.random(w.rows).astype(np.float32) + 0.05)
+        got = g.score(reduce=reduce, causal_window=int(causal), row_weight=None if rw is None else rw.cuda()).cpu().numpy()
+        ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale, mode=reduce,
+                                causal_window=causal, row_weight=None if rw is None else rw.double().numpy())
+        assert_scores_close(got, ref, g.cu)
+
+
 def test_score_token_major_key_layout_and_reproducibility(B, W, oracle):
     w = small(W, n_in=900)
     g = Gpu(B, W, w, [0, 1])
@@ -451,6 +478,38 @@ def test_specpc_exact_on_dyadic_scores(B, W, oracle):
             lens = np.diff(cu)
             np.testing.assert_array_equal(n_keep, np.minimum(lens, np.minimum(c_max, np.maximum(lens - forced, 0))
                                                              + np.minimum(forced, lens)))
+
+
+def test_specpc_seeded_random_shapes(B, W, oracle):
+    """Seeded sweep of the keep set: ragged batches with empty sequences, both reductions, max pooling
+    and the printed average-then-max order, neighbour widths, forced tails; dyadic scores keep the
+    fp32 sums and power-of-two averages exact, so the lists must be identical."""
+    rng = np.random.default_rng(99)
+    for case in range(24):
+        L, H = int(rng.integers(1, 5)), int(rng.integers(1, 4))
+        n_seq = int(rng.integers(1, 5))
+        lens = [int(rng.choice([0, 1, 3, 64, 129, 1000, int(rng.integers(1, 4000))])) for _ in range(n_seq)]
+        if sum(lens) == 0:
+            lens[-1] = 17
+        cu = [0] + list(np.cumsum(lens))
+        T = cu[-1]
+        scores = (rng.integers(0, 64, size=(L, H, T)) / 64).astype(np.float32)
+        cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda")
+        pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=64, n_lookahead=1, n_window=0,
+                            softmax_scale=1.0, total_tokens=T, n_in=max(lens), n_seq=n_seq, cu_seqlens=cu_t)
+        reduce = case % 2
+        two_stage = case % 3 == 0
+        k = int(rng.choice([1, 2, 4, 8])) if two_stage else int(rng.choice([1, 3, 7, 9]))
+        c_max = int(rng.choice([1, 5, 64, 300, 5000]))
+        nb = int(rng.choice([0, 1, 2, 8, 33]))
+        forced = int(rng.integers(0, 40)) if case % 4 == 1 or two_stage else 0
+        pool = B.POOL_AVG_THEN_MAX if two_stage else 0
+        cap = max(lens)
+        keep, n_keep = run_keep(B, pr, torch.from_numpy(scores).cuda(), reduce, pool, k, c_max, nb, forced, cap, n_seq)
+        ok, on, _, _ = oracle.specpc_select(scores.astype(np.float64), cu, reduce, oracle.POOL_AVG_THEN_MAX if two_stage else 0,
+                                            k, c_max, nb, forced, cap)
+        np.testing.assert_array_equal(n_keep, on, err_msg="case %d" % case)
+        np.testing.assert_array_equal(keep, ok, err_msg="case %d" % case)
 
 
 def test_specpc_config3_full(B, W, oracle):
