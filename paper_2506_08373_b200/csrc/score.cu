@@ -7,20 +7,26 @@
 //   merge    combines the segments' statistics into one constant per row,
 //            c_i = log2e*scale*max_i + log2 Z_i - log2 w_i;
 //   pass 2   S^T = K Q^T per tile (keys on TMEM lanes, query rows on columns):
-//            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one store per key.
+//            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one reduction per key
+//            and warpgroup.
 // Both passes are persistent, warp-specialised kernels: warp 0 feeds K tiles (and the unit's Q)
-// with TMA into a shared-memory ring, warp 1 issues tcgen05.mma into four 128-column TMEM
-// buffers, and four epilogue warpgroups (16 warps, four per SM sub-partition) drain them with
-// tcgen05.ld and do the exponentials.  The warpgroups form two pairs; a pair takes a whole
-// buffer and its two warpgroups split the buffer's columns in halves, so each pair always has a
-// second buffer being filled while it works.  The exponential is the scarce resource (16 MUFU
-// results per clock per SM against 32 logits per clock from the tensor cores), so a fixed share
-// of the elements is evaluated on the FMA pipes instead (range reduction + cubic polynomial,
-// relative error 7.5e-5), and the surrounding arithmetic uses the packed two-lane fp32
-// instructions to halve its issue slots.  Warpgroups never synchronise inside a unit: pass 1
-// writes their statistics as separate partials; in pass 2 a key tile belongs to one pair, whose
-// two warpgroups add their per-key sums into the zero-filled output with one reduction each
-// (two addends, so the result does not depend on their order).
+// with TMA into a shared-memory ring, one (pass 1) or two (pass 2) threads issue tcgen05.mma into
+// TMEM, and four epilogue warpgroups (16 warps, four per SM sub-partition) drain the
+// accumulators with tcgen05.ld and do the exponentials.
+//   pass 1: work items of 128 rows x 256 keys (two ring stages as one N = 256 operand), two
+//           256-column buffers, all 16 epilogue warps on the same buffer (64 columns each);
+//   pass 2: 128 keys x 128 rows, four 128-column buffers; the warpgroups form two pairs, each
+//           with its own issuing thread and two buffers, the pair's warpgroups split a
+//           buffer's columns in halves.
+// The exponential is the scarce resource (16 MUFU results per clock per SM against 32 logits per
+// clock from the tensor cores), so a fixed share of the elements is evaluated on the FMA pipes
+// instead (range reduction + cubic polynomial, relative error 7.5e-5), and the surrounding
+// arithmetic uses the packed two-lane fp32 instructions to halve its issue slots.  Warpgroups
+// never synchronise inside a unit: pass 1 writes their statistics as separate partials; in
+// pass 2 a key tile belongs to one pair, whose two warpgroups add their per-key sums into the
+// zero-filled output with one reduction each (two addends, so the result does not depend on
+// their order).  More query rows than fit in shared memory are scored in several launches over
+// groups of rows (ScoreParams::row0), each adding into the same output.
 // The global key-tile space (layer, KV head, sequence, tile) is cut into equal contiguous
 // ranges, one per CTA.
 //
