@@ -11,9 +11,10 @@
  * inputs are widened exactly to double; all arithmetic is double.
  *
  * Parity status: every function below is pinned by the CPU test-suite (brute
- * force on tiny inputs, closed forms, library special cases, invariants) except
- * pooling with an EVEN kernel size, whose window placement the paper does not
- * fix: "parity unpinned" for even k.
+ * force on tiny inputs, closed forms, library special cases, invariants).
+ * Pooling with an EVEN width has no centre and the paper does not say where
+ * the window sits; the window used, [j - k/2, j + k/2 - 1], is pinned to the
+ * first n outputs of the library pooling routine with padding k/2.
  */
 #include <math.h>
 #include <stdint.h>

@@ -260,7 +260,7 @@ def test_topk_clustered_keys_large_budget_and_odd_offsets(B, W, oracle):
 
 def test_topk_seeded_random_shapes_and_special_values(B, W, oracle):
     """Many small seeded cases: lengths around tile and vector edges, budgets from 1 to beyond n, odd
-    pooling widths, forced tails, and score vectors with negatives, signed zeros, infinities and
+    and even pooling widths, forced tails, and score vectors with negatives, signed zeros, infinities and
     long runs of equal values.  Max-pool selection is exact, ties to the lower position."""
     rng = np.random.default_rng(2024)
     for case in range(48):
@@ -282,7 +282,7 @@ def test_topk_seeded_random_shapes_and_special_values(B, W, oracle):
         else:
             x = np.where(rng.random((2, 2, T)) < 0.5, np.float32(0.0), np.float32(-0.0)).astype(np.float32)
             x[rng.random(x.shape) < 0.1] = 1e-30
-        k = int(rng.choice([1, 3, 5, 7, 9, 31]))
+        k = int(rng.choice([1, 2, 3, 4, 5, 7, 9, 31, 64]))        # even widths: window [j - k/2, j + k/2 - 1]
         c_max = int(rng.choice([1, 2, 16, 100, 1024, max(lens) + 3]))
         forced = int(rng.integers(0, min(c_max, 20) + 1)) if case % 3 == 0 else 0
         run_topk_case(B, W, oracle, x, cu, 0, k, c_max, forced)

@@ -259,6 +259,20 @@ def test_pool_matches_library(oracle, k):
     assert np.all(oracle.pool(x, k, oracle.POOL_MAX) >= x)
 
 
+@pytest.mark.parametrize("k", [2, 4, 8, 32, 64])
+def test_pool_even_width_matches_library_first_n_outputs(oracle, k):
+    """An even width has no centre: the library's pooling with padding k // 2 and stride 1 yields n + 1
+    outputs, and its first n are the windows [j - k/2, j + k/2 - 1] the oracle uses (zero padding and
+    divisor k for the average, -inf padding for the maximum)."""
+    g = torch.Generator().manual_seed(40 + k)
+    for n in (1, 3, k - 1, k, k + 1, 200):
+        x = torch.rand(n, generator=g, dtype=torch.float64) - 0.3
+        mx = torch.nn.functional.max_pool1d(x.view(1, 1, n), k, 1, k // 2).view(-1)[:n].numpy()
+        np.testing.assert_array_equal(oracle.pool(x.numpy(), k, oracle.POOL_MAX), mx)
+        av = torch.nn.functional.avg_pool1d(x.view(1, 1, n), k, 1, k // 2, count_include_pad=True).view(-1)[:n].numpy()
+        np.testing.assert_allclose(oracle.pool(x.numpy(), k, oracle.POOL_AVG), av, rtol=1e-12, atol=1e-15)
+
+
 def test_pool_brute_window(oracle):
     x = np.array([0.1, 0.9, 0.2, 0.3, 0.0, 0.0, 0.0, 0.0, 0.5, 0.4])
     got = oracle.pool(x, 7, oracle.POOL_MAX)
