@@ -192,10 +192,11 @@ struct TopkParams {
 //
 // One CTA per (sequence, layer, KV head) unit, any length.  The unit's scores are read once.
 // Every warp owns a contiguous range of positions and streams it on its own, kWarpStep
-// positions per step, straight from global memory into registers (16-byte loads, the next
-// step's loads in flight while the current one is processed), with no CTA-wide barrier per
-// step.  Every pooled key at or above a rising floor is counted in a shared histogram of the
-// keys' top kTopBits bits and appended, in position order, to the warp's candidate list in
+// positions per step, straight from global memory into registers (every lane loads its own
+// eight scores with two 16-byte loads, the next steps' loads in flight while the current one
+// is processed, and takes the three scores on either side from the neighbouring lanes by
+// shuffle), with no CTA-wide barrier per step.  Every pooled key at or above a rising floor is
+// counted in a shared histogram of the keys' top kTopBits bits and appended, in position order, to the warp's candidate list in
 // shared memory; the floor is the bin that holds the C-th largest key of the positions seen so
 // far and is raised at a few CTA-wide synchronisation points.  After the sweep the remaining
 // bits are resolved by radix passes over the candidates only, and the winners are written in
@@ -263,38 +264,28 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
-// The 16 scores around the 8 positions that start at x = xb: x in [xb - 4, xb + 12).
-// Positions outside [0, e) read as -infinity.
-__device__ __forceinline__ void load_window(const SweepGeom& g, int xb, float4 (&w)[4]) {
-  const int p_first = xb - 4 - g.mis;
-  if (p_first >= 0 && p_first + 15 < g.e) {
-    const float4* v = reinterpret_cast<const float4*>(g.src + p_first);
+// Four scores starting at position p_first (a multiple of four elements from a 16-byte boundary);
+// positions outside [0, e) read as -infinity.
+__device__ __forceinline__ float4 load4(const SweepGeom& g, int p_first) {
+  if (p_first >= 0 && p_first + 3 < g.e) return __ldg(reinterpret_cast<const float4*>(g.src + p_first));
+  float t[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) w[i] = __ldg(v + i);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float t[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int pp = p_first + 4 * i + q;
-        t[q] = (pp >= 0 && pp < g.e) ? __ldg(g.src + pp) : -INFINITY;
-      }
-      w[i] = make_float4(t[0], t[1], t[2], t[3]);
-    }
+  for (int q = 0; q < 4; ++q) {
+    const int pp = p_first + q;
+    t[q] = (pp >= 0 && pp < g.e) ? __ldg(g.src + pp) : -INFINITY;
   }
+  return make_float4(t[0], t[1], t[2], t[3]);
 }
 
-// Max-pool of width 7 over the window: position u pools elements u + 1 .. u + 7.
-__device__ __forceinline__ void pool_max7(const float4 (&w4)[4], float (&val)[kPerThread]) {
-  static_assert(kPerThread == 8, "the window code is written for eight positions per thread");
-  const float w[16] = {w4[0].x, w4[0].y, w4[0].z, w4[0].w, w4[1].x, w4[1].y, w4[1].z, w4[1].w,
-                       w4[2].x, w4[2].y, w4[2].z, w4[2].w, w4[3].x, w4[3].y, w4[3].z, w4[3].w};
-  float t3[13];                                            // maxima of three neighbours, shared by the windows
+// Max-pool of width 7 for a lane's eight positions from its own eight scores w (elements 0..7),
+// the three scores before them (l) and the three after them (r).
+__device__ __forceinline__ void pool_max7_halo(const float (&l)[3], const float4 (&w4)[2], const float (&r)[3], float (&val)[kPerThread]) {
+  const float x[14] = {l[0], l[1], l[2], w4[0].x, w4[0].y, w4[0].z, w4[0].w, w4[1].x, w4[1].y, w4[1].z, w4[1].w, r[0], r[1], r[2]};
+  float t3[12];
 #pragma unroll
-  for (int i = 1; i < 13; ++i) t3[i] = fmax3(w[i], w[i + 1], w[i + 2]);
+  for (int i = 0; i < 12; ++i) t3[i] = fmax3(x[i], x[i + 1], x[i + 2]);
 #pragma unroll
-  for (int u = 0; u < kPerThread; ++u) val[u] = fmax3(t3[u + 1], t3[u + 4], w[u + 7]);
+  for (int u = 0; u < kPerThread; ++u) val[u] = fmax3(t3[u], t3[u + 3], x[u + 6]);
 }
 
 // Word of bin b in the top-bits histogram: every lane of a warp scans 256 consecutive bins
@@ -512,20 +503,55 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     };
 
     if (max7) {
-      // two steps of loads in flight per thread; a window's registers are refilled as soon as
-      // it has been pooled
-      float4 wa[4], wb[4];
-      load_window(g, x_warp, wa);
-      if (g.n_steps > 1) load_window(g, x_warp + kWarpStep, wb);
-      for (int st = 0; st < g.n_steps; st += 2) {
-        float val[kPerThread];
-        pool_max7(wa, val);
-        if (st + 2 < g.n_steps) load_window(g, x_warp + (st + 2) * kWarpStep, wa);
-        process(val, x_warp + st * kWarpStep - g.mis, st);
-        if (st + 1 < g.n_steps) {
-          pool_max7(wb, val);
-          if (st + 3 < g.n_steps) load_window(g, x_warp + (st + 3) * kWarpStep, wb);
-          process(val, x_warp + (st + 1) * kWarpStep - g.mis, st + 1);
+      // Every lane loads its own eight scores of a step (two 16-byte loads, kAhead steps in
+      // flight); the three scores on either side come from the neighbouring lanes by shuffle.
+      // Lane 0 takes them from lane 31 of the warp's previous step (kept in `carry`; before the
+      // first step they are loaded), lane 31 loads the four scores that follow its own.
+      constexpr int kAhead = 2;                            // steps in flight (three or four spill under the 64-register cap)
+      float4 w[kAhead][2];
+#pragma unroll
+      for (int sidx = 0; sidx < kAhead; ++sidx) {
+        if (sidx < g.n_steps) {
+          const int pf = x_warp + sidx * kWarpStep - g.mis;
+          w[sidx][0] = load4(g, pf);
+          w[sidx][1] = load4(g, pf + 4);
+        }
+      }
+      float carry[3];
+      {
+        const int pb = warp * g.span - g.mis - 3;            // the three positions before my warp's range
+#pragma unroll
+        for (int q = 0; q < 3; ++q) carry[q] = (pb + q >= 0 && pb + q < e) ? __ldg(src + pb + q) : -INFINITY;
+      }
+      for (int st = 0; st < g.n_steps; st += kAhead) {
+#pragma unroll
+        for (int sidx = 0; sidx < kAhead; ++sidx) {
+          if (st + sidx < g.n_steps) {                       // warp-uniform
+            const int pf = x_warp + (st + sidx) * kWarpStep - g.mis;    // my first position
+            const float4 (&cur)[2] = w[sidx];
+            float4 after = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lane == 31) after = load4(g, pf + 8);
+            float l[3], r[3];
+            l[0] = __shfl_up_sync(0xffffffffu, cur[1].y, 1);
+            l[1] = __shfl_up_sync(0xffffffffu, cur[1].z, 1);
+            l[2] = __shfl_up_sync(0xffffffffu, cur[1].w, 1);
+            r[0] = __shfl_down_sync(0xffffffffu, cur[0].x, 1);
+            r[1] = __shfl_down_sync(0xffffffffu, cur[0].y, 1);
+            r[2] = __shfl_down_sync(0xffffffffu, cur[0].z, 1);
+            if (lane == 0) { l[0] = carry[0]; l[1] = carry[1]; l[2] = carry[2]; }
+            if (lane == 31) { r[0] = after.x; r[1] = after.y; r[2] = after.z; }
+            carry[0] = __shfl_sync(0xffffffffu, cur[1].y, 31);
+            carry[1] = __shfl_sync(0xffffffffu, cur[1].z, 31);
+            carry[2] = __shfl_sync(0xffffffffu, cur[1].w, 31);
+            float val[kPerThread];
+            pool_max7_halo(l, cur, r, val);
+            if (st + sidx + kAhead < g.n_steps) {
+              const int pn = pf + kAhead * kWarpStep;
+              w[sidx][0] = load4(g, pn);
+              w[sidx][1] = load4(g, pn + 4);
+            }
+            process(val, pf, st + sidx);
+          }
         }
       }
     } else {
