@@ -366,6 +366,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     // ---- the sweep.  The take-th largest key of the positions seen so far can only be below
     // that of the whole unit, so the bin that holds it is a floor: keys under it are out.
     uint32_t floor_key = 0;
+    uint32_t early_floor = 0;                                // highest floor taken from a part of the unit
     int cnt = 0;                                             // entries in my warp's list (warp-uniform)
     const int x_warp = warp * g.span + lane * kPerThread;
 
@@ -494,11 +495,23 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
         n_pend += n_hot;
         __syncwarp();
       }
-      if (((st + 1) & st) == 0 || (st & 31) == 31) expand();  // the histogram must be complete for the floor
-      if (((st + 1) & st) == 0 || (st & 31) == 31) {       // after steps 0, 1, 3, 7, 15, 31, then every 32nd
+      // Floor updates after steps 0, 1, 3, 7, 15, 31, then every 32nd; none after the last step, the
+      // final selection follows it anyway.
+      const bool refloor = (((st + 1) & st) == 0 || (st & 31) == 31) && st + 1 < g.n_steps;
+      if (refloor) expand();                                 // the histogram must be complete for the floor
+      if (refloor) {
+        // While only a fraction f of the unit has been seen, the floor is taken at rank 2 f take + 64
+        // of the keys seen instead of rank take: about f take of them are expected above the final
+        // threshold, so this bin is below it unless the large keys crowd into the part seen first.
+        // That case leaves fewer than `take` candidates at the end, which the final selection
+        // detects and hands to the generic path; the result is exact either way.
         int fb, ab;
-        if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, fb, ab))
+        const long long seen = (long long)(st + 1) * (kWarpStep * kSelWarps);
+        const int need = seen >= e ? take : min(take, (int)(2 * ((long long)take * seen / e)) + 64);
+        if (locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, need, wsum, out2, fb, ab)) {
           floor_key = max(floor_key, (uint32_t)fb << (32 - kTopBits));
+          early_floor = max(early_floor, (uint32_t)fb << (32 - kTopBits));    // the same in every thread of the CTA
+        }
       }
     };
 
@@ -568,8 +581,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
     expand();
     if (lane == 0) wcnt[warp] = cnt;
     int b1 = 0, above = 0;
-    bool fits = locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails only on NaN scores
-    fits = fits && *overflow == 0;
+    bool fits = locate_bin(top_hist + top_word(tid * (kTopBins / kSelThreads)), kTopBins / kSelThreads, take, wsum, out2, b1, above);   // fails on NaN scores or when an early floor was too high
+    // Below an early floor the histogram and the lists are incomplete: a threshold bin found there
+    // means that floor was too high.
+    fits = fits && *overflow == 0 && ((uint32_t)b1 << (32 - kTopBits)) >= early_floor;
     if (fits) {
       // ---- remaining bits on the candidates only (every warp walks its own list)
       int known = kTopBits;

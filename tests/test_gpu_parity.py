@@ -258,6 +258,27 @@ def test_topk_clustered_keys_large_budget_and_odd_offsets(B, W, oracle):
     run_topk_case(B, W, oracle, scores, [0, 4099, 4099 + 33333, 4099 + 33333 + 12345], 0, 7, 512, 40)
 
 
+def test_topk_large_keys_crowded_into_the_part_swept_first(B, W, oracle):
+    """The sweep raises its floor early from the part of the unit seen so far.  Here that part (the first
+    256 positions of each of the 16 ranges the warps stream) holds a third of the large keys, so the early
+    floor lands above the final threshold and most winners, met later, fall under it: the kernel must
+    notice and still return the exact set."""
+    rng = np.random.default_rng(11)
+    n, c_max = 100000, 2048
+    x = (rng.random((1, 2, n)) * 0.01).astype(np.float32)
+    span = 6400                                               # ceil(n / 16 / 256) * 256
+    first = np.concatenate([np.arange(w * span, w * span + 256) for w in range(16)])
+    first = first[first < n]
+    early = rng.choice(first, 1000, replace=False)
+    late = rng.choice(np.setdiff1d(np.arange(n), first), 3000, replace=False)
+    for h in range(2):
+        x[0, h, early] = (10.0 * 2.0 ** (3.0 * rng.random(early.size))).astype(np.float32)
+        x[0, h, late] = (10.0 * 2.0 ** (3.0 * rng.random(late.size))).astype(np.float32)
+    for k in (1, 7):
+        run_topk_case(B, W, oracle, x, [0, n], 0, k, c_max, 0)
+    run_topk_case(B, W, oracle, x, [0, n], 0, 7, 512, 0)
+
+
 def test_topk_seeded_random_shapes_and_special_values(B, W, oracle):
     """Many small seeded cases: lengths around tile and vector edges, budgets from 1 to beyond n, odd
     and even pooling widths, forced tails, and score vectors with negatives, signed zeros, infinities and
