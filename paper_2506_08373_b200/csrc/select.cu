@@ -495,9 +495,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) pool_topk_kernel(TopkParams p)
         n_pend += n_hot;
         __syncwarp();
       }
-      // Floor updates after steps 0, 1, 3, 7, 15, 31, then every 32nd; none after the last step, the
+      // Floor updates after steps 0, 3, 15, 63, then every 64th; none after the last step, the
       // final selection follows it anyway.
-      const bool refloor = (((st + 1) & st) == 0 || (st & 31) == 31) && st + 1 < g.n_steps;
+      const bool refloor = ((((st + 1) & st) == 0 && (__popc(st) & 1) == 0) || (st & 63) == 63) && st + 1 < g.n_steps;
       if (refloor) expand();                                 // the histogram must be complete for the floor
       if (refloor) {
         // While only a fraction f of the unit has been seen, the floor is taken at rank 2 f take + 64
