@@ -736,7 +736,29 @@ __global__ void __launch_bounds__(kSelThreads) specpc_keep_kernel(KeepParams p) 
     key.e = e; key.pool = p.pool; key.k = p.pool_k;
     key.keys = nullptr;
     if (e <= p.cap) {
-      for (int j = tid; j < e; j += kSelThreads) keys[j] = key(j);
+      if (p.pool == SPEC_POOL_MAX && p.pool_k == 7) {
+        // width-7 maximum with the loads of eight positions per thread in flight at once;
+        // positions outside [0, e) read as -infinity
+        const float* src = p.tok + begin;
+        for (int j0 = tid; j0 < e; j0 += 8 * kSelThreads) {
+          float w[8][7];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int t = 0; t < 7; ++t) {
+              const int q = j0 + u * kSelThreads + t - 3;
+              w[u][t] = (q >= 0 && q < e) ? __ldg(src + q) : -INFINITY;
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * kSelThreads;
+            if (j < e) keys[j] = to_key(fmax3(fmax3(w[u][0], w[u][1], w[u][2]), fmax3(w[u][3], w[u][4], w[u][5]), w[u][6]));
+          }
+        }
+      } else {
+        for (int j = tid; j < e; j += kSelThreads) keys[j] = key(j);
+      }
       key.keys = keys;
       __syncthreads();
     }
