@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC = {
     # workload index -> {kernel group: (bytes per layer, source file, source hash)}
     1: {"score": ((138.78e6 + 7.37e6 + 140.94e6 + 1.41e6) / 4, "score.cu", "c6454076e2803746")},
-    2: {"select": (33.67e6 / 8, "select.cu", "67867e7027b3d2e4"),
+    2: {"select": (33.67e6 / 8, "select.cu", "08ec50023cb8d667"),
         "gather": ((67.69e6 + 16.88e6) / 8, "compact.cu", "08fc6f03baf192d3")},
 }
 

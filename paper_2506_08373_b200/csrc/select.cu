@@ -762,11 +762,80 @@ __global__ void __launch_bounds__(kSelThreads) specpc_keep_kernel(KeepParams p) 
       key.keys = keys;
       __syncthreads();
     }
-    uint32_t T;
-    int need_eq;
-    radix_select(key, e, take, sc, T, need_eq);
     const int nb = p.n_neighbor;
-    ordered_emit(key, e, T, need_eq, sc, [&](int, int j) { mark(max(j - nb, 0), min(j + nb, e - 1)); });
+    if (key.keys) {
+      // Resident keys: three radix passes (11, 11, 10 bits) find the key T of the take-th largest
+      // position.  Thread t looks at positions t, t + 512, ..., so the lanes of a warp hold
+      // consecutive positions and the runs of equal digits that pooling produces are merged into
+      // one histogram update by ballot.  Marking needs no order for keys above T; of the keys
+      // equal to T the first need_eq by position are found with a scan over the warps' ballots.
+      uint32_t* hist = sc.hist;
+      int* out2 = sc.misc;
+      int* wsum = sc.misc + 8;
+      const uint32_t lt_mask = (1u << lane) - 1u;
+      const int rows = (e + kSelThreads - 1) / kSelThreads;
+      uint32_t prefix = 0, mask = 0;
+      int remaining = take;
+#pragma unroll 1
+      for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
+        const int bins = pass == 2 ? 1024 : 2048;
+        for (int b = tid; b < bins; b += kSelThreads) hist[b] = 0;
+        __syncthreads();
+        for (int i = 0; i < rows; ++i) {
+          const int j = i * kSelThreads + tid;
+          const uint32_t kk = j < e ? keys[j] : 0u;
+          const bool in = j < e && (kk & mask) == prefix;
+          const uint32_t dg = (kk >> shift) & (uint32_t)(bins - 1);
+          const uint32_t dg_prev = __shfl_up_sync(0xffffffffu, dg, 1);
+          const uint32_t ins = __ballot_sync(0xffffffffu, in);
+          const bool head = in && (lane == 0 || !((ins >> (lane - 1)) & 1u) || dg_prev != dg);
+          const uint32_t heads = __ballot_sync(0xffffffffu, head);
+          if (head) {
+            const uint32_t stop = (heads | ~ins) & ~(lt_mask | (1u << lane));   // next run, or a lane that is out
+            atomicAdd(&hist[dg], (uint32_t)((stop ? __ffs(stop) - 1 : 32) - lane));
+          }
+        }
+        int dg, ab;
+        locate_bin(hist + tid * (bins / kSelThreads), bins / kSelThreads, remaining, wsum, out2, dg, ab);
+        remaining -= ab;
+        prefix |= (uint32_t)dg << shift;
+        mask |= (uint32_t)(bins - 1) << shift;
+      }
+      const uint32_t T = prefix;
+      const int need_eq = remaining;
+      uint32_t* eqm = sc.hist;                               // [rows][kSelWarps] ballots of the keys equal to T
+      for (int i = 0; i < rows; ++i) {
+        const int j = i * kSelThreads + tid;
+        const uint32_t kk = j < e ? keys[j] : 0u;
+        if (j < e && kk > T) mark(max(j - nb, 0), min(j + nb, e - 1));
+        const uint32_t be = __ballot_sync(0xffffffffu, j < e && kk == T);
+        if (lane == 0) eqm[i * kSelWarps + warp] = be;
+      }
+      __syncthreads();
+      const int n_ent = rows * kSelWarps;
+      const int ept = (n_ent + kSelThreads - 1) / kSelThreads;
+      const int e0 = tid * ept, e1 = min(e0 + ept, n_ent);
+      int mine = 0;
+      for (int en = e0; en < e1; ++en) mine += __popc(eqm[en]);
+      int total_eq;
+      int before = block_exclusive_scan(mine, wsum + kSelWarps, total_eq);
+      for (int en = e0; en < e1 && before < need_eq; ++en) {
+        uint32_t bits = eqm[en];
+        const int base = (en / kSelWarps) * kSelThreads + (en % kSelWarps) * 32;
+        while (bits && before < need_eq) {
+          const int j = base + __ffs(bits) - 1;
+          bits &= bits - 1;
+          mark(max(j - nb, 0), min(j + nb, e - 1));
+          ++before;
+        }
+      }
+    } else {
+      uint32_t T;
+      int need_eq;
+      radix_select(key, e, take, sc, T, need_eq);
+      ordered_emit(key, e, T, need_eq, sc, [&](int, int j) { mark(max(j - nb, 0), min(j + nb, e - 1)); });
+    }
   } else if (take > 0) {
     for (int w = tid; w < ((e + 31) >> 5); w += kSelThreads) {
       const int hi = min(e - 1, (w << 5) + 31);
