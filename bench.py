@@ -237,7 +237,7 @@ class State:
                 events[3].record()
         else:
             B.spec_pool_topk(self.pr, self.scores, B.POOL_MAX, w.pool_k, w.c_max, 0, self.idx, self.cnt,
-                             status_word=self.status)
+                             workspace=self.ws, status_word=self.status)
             if events is not None:
                 events[2].record()
             if self.bt is not None:

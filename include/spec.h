@@ -49,8 +49,7 @@ typedef enum {
   SPEC_ERR_UNSUPPORTED = -3,    /* shape outside the implemented range, or not an sm_100 device */
   SPEC_ERR_WORKSPACE = -4,      /* workspace NULL or smaller than spec_workspace_bytes() */
   SPEC_ERR_CUDA = -5,           /* a CUDA runtime / driver call failed */
-  SPEC_ERR_TIMEOUT = -6,        /* device side: a bounded wait expired (status_word only) */
-  SPEC_ERR_NOT_IMPLEMENTED = -7
+  SPEC_ERR_TIMEOUT = -6         /* device side: a bounded wait expired (status_word only) */
 } spec_status;
 
 /* Reduction over query rows (spec_score) or over layers and heads (specpc_token_select). */
@@ -75,7 +74,12 @@ typedef enum {
  * owns tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (n_s of them; cu_seqlens is a
  * DEVICE array of n_seq+1 non-decreasing int32 with cu_seqlens[n_seq] <=
  * total_tokens).  cu_seqlens == NULL means one sequence covering tokens
- * [0, n_in).  Element (layer, kv_head, token, c) of K is at
+ * [0, n_in).  With cu_seqlens given, the sequence lengths are only known on
+ * the device; n_in is then the caller's upper bound on every n_s (it sizes
+ * shared memory and picks launch shapes; 0 = no bound known, total_tokens is
+ * assumed).  A sequence longer than a non-zero bound is not processed: the
+ * selection calls report SPEC_ERR_BAD_ARG in status_word and return empty
+ * lists for it.  Element (layer, kv_head, token, c) of K is at
  *   k + layer*k_stride_layer + kv_head*k_stride_head + token*k_stride_token + c
  * (strides in elements, bf16; the head_dim axis is contiguous); V likewise.
  * K/V base pointers and strides*2 bytes must be multiples of 16 bytes.
@@ -83,7 +87,7 @@ typedef enum {
 typedef struct {
   int32_t n_seq;                /* >= 1 (<= 1024) */
   const int32_t* cu_seqlens;    /* device [n_seq+1] or NULL */
-  int32_t n_in;                 /* used only when cu_seqlens == NULL */
+  int32_t n_in;                 /* cu_seqlens == NULL: the prompt length; else an upper bound of every n_s, or 0 */
   int32_t total_tokens;         /* T */
   int32_t n_layers, n_q_heads, n_kv_heads, head_dim;   /* head_dim in {64, 128}; n_q_heads % n_kv_heads == 0 */
   int32_t n_lookahead, n_window;                        /* R >= 1; n_lookahead may be 0 (SnapKV special case) */
@@ -142,10 +146,35 @@ int32_t spec_score(const spec_problem* problem, const void* q, const void* k, co
  *             padded with -1 when fewer than c_max positions exist
  *  count_out  optional [n_seq, n_layers, n_kv_heads] int32 number of valid entries
  * Requires 1 <= pool_k <= 255, 0 <= n_forced_tail <= c_max, c_max >= 1.
+ * workspace is optional (NULL, 0): the lists are the same either way.  With a workspace of
+ * spec_workspace_bytes() the default pooling (SPEC_POOL_MAX, pool_k = 7) takes its fastest path,
+ * which parks candidate positions there.
  */
 int32_t spec_pool_topk(const spec_problem* problem, const float* scores, int32_t pool, int32_t pool_k,
                        int32_t c_max, int32_t n_forced_tail, int32_t* idx_out, int32_t* count_out,
                        void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
+
+/*
+ * Cache indices and vertical indices from one sweep -- Algorithm 1 lines 10, 11 and 13.
+ *
+ * Sparse prefill wants two index sets from the same pooled scores of a head: i_cache (line 13,
+ * exactly what spec_pool_topk returns for c_max and n_forced_tail) and i_vert = topk(s, n_vert)
+ * (line 11; the hyper-parameter table uses n_vert = 2048), the key columns every query attends
+ * to in a Vertical-Slash kernel.  This call reads and pools the scores once and selects both
+ * budgets from the resident pooled keys.  i_vert is taken over the eligible positions [0, e)
+ * only (in Algorithm 1 the window keys carry no score); no tail is appended to it.
+ *
+ *  idx_out, count_out        as in spec_pool_topk
+ *  vert_idx_out              [n_seq, n_layers, n_kv_heads, n_vert] int32, ascending sequence-local
+ *                            positions (one sorted int32 list per head, the form a Vertical-Slash
+ *                            kernel takes its vertical indices in), padded with -1
+ *  vert_count_out            optional [n_seq, n_layers, n_kv_heads] int32, min(n_vert, e)
+ * Requires n_vert >= 1 and the argument rules of spec_pool_topk (workspace optional, as there).
+ */
+int32_t spec_pool_topk_vert(const spec_problem* problem, const float* scores, int32_t pool, int32_t pool_k,
+                            int32_t c_max, int32_t n_forced_tail, int32_t* idx_out, int32_t* count_out,
+                            int32_t n_vert, int32_t* vert_idx_out, int32_t* vert_count_out,
+                            void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream);
 
 /*
  * K/V compaction -- Algorithm 1 line 15 (cache <- K[i_cache], V[i_cache]).
@@ -178,8 +207,8 @@ int32_t spec_compact_kv(const spec_problem* problem, const void* k, const void* 
  *  keep_out    [n_seq, keep_capacity] int32, ascending, padded with -1
  *  n_keep_out  [n_seq] int32
  * keep_capacity must be >= min(max_len, c_max*(2*n_neighbor+1) + n_forced_tail) where max_len is
- * n_in (cu_seqlens == NULL) or total_tokens (with SPEC_POOL_AVG_THEN_MAX: min(max_len, c_max +
- * n_forced_tail)); else SPEC_ERR_BAD_ARG.
+ * n_in when it is given (see spec_problem) and total_tokens otherwise (with
+ * SPEC_POOL_AVG_THEN_MAX: min(max_len, c_max + n_forced_tail)); else SPEC_ERR_BAD_ARG.
  */
 int32_t specpc_token_select(const spec_problem* problem, const float* scores, int32_t layer_head_reduce,
                             int32_t pool, int32_t pool_k, int32_t c_max, int32_t n_neighbor,
@@ -227,12 +256,17 @@ int32_t spec_gather_tokens(const spec_problem* problem, const void* k, const voi
  *     limit).  The array costs SPEC_STATIC_MAX_TOKENS * 4 bytes (1 MiB) of device memory on
  *     every GPU that loads the library, for the life of the process.
  *   - The first call on each device looks up the array's device address (with that device
- *     current).  Make that first call outside any stream capture.
+ *     current).  Make that first call outside any stream capture.  The array itself comes into
+ *     being when the library's device code is first loaded on a device, which may be that same
+ *     first call: make it before a memory pool claims the rest of the device.  The address is
+ *     remembered per device; after cudaDeviceReset it is stale and the process must not call
+ *     this entry point again.
+ *   - SPEC_POOL_AVG_THEN_MAX is not offered (it needs a second vector): SPEC_ERR_UNSUPPORTED.
  *   - All calls on a device share the one array.  It keeps whatever the last call left there;
  *     each call rewrites every element it later reads, so results never depend on earlier
  *     calls -- but two calls that overlap on the GPU (different streams, no dependency) race
  *     on it.  Order them.
- * Arguments and results are exactly those of specpc_token_select, minus the workspace.
+ * Otherwise arguments and results are those of specpc_token_select, minus the workspace.
  */
 #define SPEC_STATIC_MAX_TOKENS 262144
 int32_t specpc_token_select_static(const spec_problem* problem, const float* scores, int32_t layer_head_reduce,

@@ -12,13 +12,12 @@ import torch
 from . import build as _build
 
 SPEC_OK = 0
-ERR_BAD_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_IMPLEMENTED = \
-    -1, -2, -3, -4, -5, -6, -7
+ERR_BAD_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 REDUCE_SUM, REDUCE_MAX = 0, 1
 POOL_MAX, POOL_AVG, POOL_AVG_THEN_MAX = 0, 1, 2
 
-EXPORTS = ("spec_workspace_bytes", "spec_last_error", "spec_score", "spec_pool_topk", "spec_compact_kv",
-           "specpc_token_select", "spec_gather_tokens", "specpc_token_select_static")
+EXPORTS = ("spec_workspace_bytes", "spec_last_error", "spec_score", "spec_pool_topk", "spec_pool_topk_vert",
+           "spec_compact_kv", "specpc_token_select", "spec_gather_tokens", "specpc_token_select_static")
 STATIC_MAX_TOKENS = 262144
 
 
@@ -61,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.spec_score.argtypes = [pp, vp, vp, vp, i32, i32, vp, vp, sz, vp, vp]
         L.spec_pool_topk.restype = i32
         L.spec_pool_topk.argtypes = [pp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+        L.spec_pool_topk_vert.restype = i32
+        L.spec_pool_topk_vert.argtypes = [pp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
         L.spec_compact_kv.restype = i32
         L.spec_compact_kv.argtypes = [pp, vp, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp]
         L.specpc_token_select.restype = i32
@@ -133,6 +134,14 @@ def spec_pool_topk(problem, scores, pool, pool_k, c_max, n_forced_tail, idx_out,
     wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().spec_pool_topk(ctypes.byref(problem), _ptr(scores), pool, pool_k, c_max, n_forced_tail,
                                 _ptr(idx_out), _ptr(count_out), _ptr(workspace), wsb, _ptr(status_word), _stream()))
+
+
+def spec_pool_topk_vert(problem, scores, pool, pool_k, c_max, n_forced_tail, idx_out, count_out, n_vert,
+                        vert_idx_out, vert_count_out=None, workspace=None, status_word=None):
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().spec_pool_topk_vert(ctypes.byref(problem), _ptr(scores), pool, pool_k, c_max, n_forced_tail,
+                                     _ptr(idx_out), _ptr(count_out), n_vert, _ptr(vert_idx_out), _ptr(vert_count_out),
+                                     _ptr(workspace), wsb, _ptr(status_word), _stream()))
 
 
 def spec_compact_kv(problem, k, v, idx, c_max, k_out, v_out, block_table=None, page_size=0, n_pages=0,

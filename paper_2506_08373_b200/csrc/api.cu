@@ -24,6 +24,8 @@ int check_problem(const spec_problem* p) {
     if (p->n_seq != 1) return fail(SPEC_ERR_BAD_ARG, "cu_seqlens is NULL but n_seq=%d", p->n_seq);
     if (p->n_in < 0 || p->n_in > p->total_tokens)
       return fail(SPEC_ERR_BAD_ARG, "n_in=%d outside [0, total_tokens=%d]", p->n_in, p->total_tokens);
+  } else if (p->n_in < 0) {
+    return fail(SPEC_ERR_BAD_ARG, "n_in=%d is negative (with cu_seqlens it is an upper bound of the sequence lengths, or 0)", p->n_in);
   }
   if (p->n_layers < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1)
     return fail(SPEC_ERR_BAD_ARG, "n_layers, n_q_heads and n_kv_heads must be >= 1");
@@ -91,6 +93,15 @@ WorkspacePlan plan_workspace(const spec_problem* p) {
   w.token_off = off;
   w.token_bytes = 2 * (size_t)(p->total_tokens > 0 ? p->total_tokens : 1) * sizeof(float);   // token scores, and their average pool
   off = align_up(off + w.token_bytes, 256);
+  w.sel_head_off = off;
+  w.sel_head_words = 4 + max_seq_len(p) / kSelChunkMin + 2;
+  w.sel_head_bytes = (size_t)n_units * w.sel_head_words * sizeof(int32_t);
+  off = align_up(off + w.sel_head_bytes, 256);
+  // candidates of sequence s of a row start at entry cu[s] + s*kSelCandSlack and may fill n_s + kSelCandSlack entries
+  w.sel_row_entries = (((int64_t)p->total_tokens + 1) & ~(int64_t)1) + (int64_t)p->n_seq * kSelCandSlack + 8;
+  w.sel_cand_off = off;
+  w.sel_cand_bytes = (size_t)w.sel_row_entries * (size_t)p->n_layers * p->n_kv_heads * 8;
+  off = align_up(off + w.sel_cand_bytes, 256);
   w.total = off;
   return w;
 }

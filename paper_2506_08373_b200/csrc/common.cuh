@@ -34,9 +34,19 @@ struct WorkspacePlan {
   size_t partial_off, partial_bytes;   // per-segment row statistics (pass 1)
   size_t rowc_off, rowc_bytes;         // per-row softmax constants
   size_t token_off, token_bytes;       // SpecPC token scores (two vectors of total_tokens floats)
+  size_t sel_head_off, sel_head_bytes; // streaming selection: sel_head_words words per (sequence, layer, KV head) unit
+  int sel_head_words;                  // four words, then one candidate count per chunk
+  size_t sel_cand_off, sel_cand_bytes; // streaming selection: candidate (key, position) pairs
+  int64_t sel_row_entries;             // candidate entries per (layer, KV head) row
   size_t total;
 };
 SPEC_HIDDEN WorkspacePlan plan_workspace(const spec_problem* p);
+// Streaming selection: every chunk of a sequence owns a segment of the candidate array as long as
+// the chunk itself (at most kSelChunkMax positions, at least kSelChunkMin), so a sequence needs
+// its length plus a partial chunk; the chunks' candidate counts sit in the unit's header.
+constexpr int kSelChunkMax = 4096;
+constexpr int kSelChunkMin = 1024;
+constexpr int kSelCandSlack = 2 * kSelChunkMax;
 
 #define SPEC_CUDA_OK(expr)                                                              \
   do {                                                                                  \

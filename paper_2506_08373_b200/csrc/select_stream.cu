@@ -1,0 +1,533 @@
+// Streaming pool + top-C selection for the default pooling (Algorithm 1 lines 10, 11 and 13 with
+// the hyper-parameter table's Max pool of width 7), used when the caller provides a workspace.
+//
+// Three kernels on the caller's stream; no CTA ever waits for another:
+//   1. sample_floor_kernel, one CTA per (sequence, layer, KV head) unit: pools one 32-byte sector
+//      out of every 32..128 positions (a sector holds the whole width-7 window of its fourth
+//      score) and takes, from a two-level histogram of the sampled keys (top 11 bits, then the
+//      next 11), the key a few standard deviations below the rank the budget corresponds to.
+//      That key is a floor under the final threshold with overwhelming probability, and it does
+//      not depend on where in the unit the large scores sit (rising, falling or concentrated
+//      scores cost the same).
+//   2. stream_sweep_kernel, one small CTA per (unit, chunk of 4096 positions), eight to an SM: the
+//      chunk is staged in shared memory with one bulk asynchronous copy and pooled from there
+//      (three 16-byte reads per four positions, nothing written back); the positions at or above
+//      the floor go, as (key, position) pairs, to the chunk's own segment of the unit's candidate
+//      array in the workspace.  The scores are read from global memory once.
+//   3. stream_finish_kernel, one CTA per unit: three radix passes (11 + 11 + 10 bits) over the
+//      candidates, held in shared memory, find the exact threshold key; winners and ties are
+//      marked in position bitmaps and written out in ascending position, ties to the lower
+//      position.  A second budget (the vertical indices) is selected from the same candidates.
+// If the floor was too high or too low for the candidate array (fewer candidates than the budget,
+// or more than fit: only with massively tied scores), the finishing CTA falls back to the generic
+// selection that recomputes pooled keys from global memory.  The result is exact in every case.
+#include "select_common.cuh"
+
+#include <algorithm>
+
+namespace spec {
+
+constexpr int kStreamBins = 2048;
+constexpr int kSweepThreads = 128;
+constexpr int kSweepWarps = kSweepThreads / 32;
+constexpr int kMaxStepsPerWarp = 8;              // 128-position steps a sweeping warp keeps in registers
+constexpr int kMaxSamples = 4096;
+constexpr uint32_t kNoSelection = 0xFFFFFFFFu;   // floor value of a unit that keeps everything or nothing
+
+struct StreamParams {
+  const float* scores;
+  const int32_t* cu;
+  int64_t T;
+  int n_in, L, H, n_forced, c_max, n_vert;
+  int chunk;                  // positions per sweeping CTA (multiple of 128)
+  int chunks_max;             // CTAs per unit
+  int bitmap_words;           // words of one position bitmap of the finishing CTA
+  int max_len;                // the host's bound on any sequence length (sizes the grid and shared memory)
+  int held_cap;               // candidates the finishing CTA can hold in shared memory
+  int32_t* head;              // [units][head_words]: floor key, unused, unused, failure flag, then a candidate count per chunk
+  int head_words;
+  uint2* cand;                // candidate (key, position) pairs
+  int64_t row_entries;        // candidate entries per (layer, KV head) row
+  int32_t* idx_out;
+  int32_t* count_out;
+  int32_t* vert_out;
+  int32_t* vert_count_out;
+  int32_t* status;
+};
+
+struct UnitGeom {
+  int s, l, h, begin, n, forced, e;
+  bool over;                  // longer than the host's bound: treated as empty and reported
+  int take[2];
+  const float* src;
+  int64_t cand_off;
+  int cand_cap;
+};
+
+__device__ __forceinline__ UnitGeom unit_geom(const StreamParams& p, int unit) {
+  UnitGeom g;
+  g.h = unit % p.H;
+  g.l = (unit / p.H) % p.L;
+  g.s = unit / (p.H * p.L);
+  seq_range(p.cu, p.n_in, g.s, g.begin, g.n);
+  g.over = g.n > p.max_len;
+  if (g.over) g.n = 0;
+  g.forced = min(p.n_forced, g.n);
+  g.e = g.n - g.forced;
+  g.take[0] = max(min(p.c_max - g.forced, g.e), 0);
+  g.take[1] = max(min(p.n_vert, g.e), 0);
+  g.src = p.scores + ((int64_t)g.l * p.H + g.h) * p.T + g.begin;
+  // even, so that a segment starts on a 16-byte boundary
+  g.cand_off = ((int64_t)g.l * p.H + g.h) * p.row_entries + ((g.begin + 1) & ~1) + (int64_t)g.s * kSelCandSlack;
+  g.cand_cap = g.n + kSelCandSlack;
+  return g;
+}
+
+__device__ __forceinline__ float key_to_float(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// ---------------------------------------------------------------- 1. the floor -------
+
+__global__ void __launch_bounds__(kSelThreads) sample_floor_kernel(const StreamParams p) {
+  __shared__ uint32_t hist[kStreamBins];
+  __shared__ uint32_t skey[kMaxSamples];
+  __shared__ int wsum[32];
+  __shared__ int out2[4];
+  const int unit = blockIdx.x, tid = threadIdx.x;
+  const UnitGeom g = unit_geom(p, unit);
+  const int tk = max(g.take[0], g.take[1]);
+  const bool selects = (g.take[0] > 0 && g.take[0] < g.e) || (g.take[1] > 0 && g.take[1] < g.e);
+  uint32_t floor_key = kNoSelection;
+  if (selects) {
+    floor_key = 0;
+    for (int b = tid; b < kStreamBins; b += kSelThreads) hist[b] = 0;
+    // x = position + mis8 puts every multiple of eight on a 32-byte boundary of global memory
+    const int mis8 = (int)((reinterpret_cast<uintptr_t>(g.src) >> 2) & 7u);
+    const int X = g.e + mis8;
+    int shift = g.e >= 65536 ? 7 : g.e >= 16384 ? 6 : 5;             // one sample per 2^shift positions
+    while (((X >> shift) + 1) > kMaxSamples) ++shift;
+    const int spg = 1 << (shift - 3);                                // sectors per sample group
+    const int n_sectors = (X + 7) >> 3;
+    const int n_groups = (n_sectors + spg - 1) / spg;                // <= kMaxSamples
+    __syncthreads();
+    for (int m = tid; m < n_groups; m += kSelThreads) {
+      uint32_t hsh = ((uint32_t)unit * 0x9E3779B1u) ^ ((uint32_t)m * 0x85EBCA6Bu);
+      hsh ^= hsh >> 15; hsh *= 0x2C1B3C6Du; hsh ^= hsh >> 12;
+      const int q = m * spg + (int)(hsh % (uint32_t)min(spg, n_sectors - m * spg));
+      const int p0 = q * 8 - mis8;                                   // position of the sector's first score
+      const int centre = p0 + 3;
+      uint32_t key = 0;                                              // 0: no sample here (below every real key's top bits)
+      if (centre >= 0 && centre < g.e) {
+        float v[8];
+        if (p0 >= 0 && p0 + 8 <= g.e) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(g.src + p0));
+          const float4 b = __ldg(reinterpret_cast<const float4*>(g.src + p0 + 4));
+          v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = (p0 + i >= 0 && p0 + i < g.e) ? __ldg(g.src + p0 + i) : -INFINITY;
+        }
+        key = to_key(fmax3(fmax3(v[0], v[1], v[2]), fmax3(v[3], v[4], v[5]), v[6]));   // pooled value of the centre
+        atomicAdd(&hist[key >> 21], 1u);
+      }
+      skey[m] = key;
+    }
+    // About tk / 2^shift of the samples lie above the threshold; the floor is taken four standard
+    // deviations further down the sample.
+    const float m_exp = (float)tk / (float)(1 << shift);
+    const int rho = (int)(m_exp + 4.f * sqrtf(m_exp) + 8.f);
+    int fb, ab;
+    if (locate_bin(hist + tid * (kStreamBins / kSelThreads), kStreamBins / kSelThreads, rho, wsum, out2, fb, ab)) {
+      // second level: the next 11 bits among the samples of that bin
+      for (int b = tid; b < kStreamBins; b += kSelThreads) hist[b] = 0;
+      __syncthreads();
+      for (int m = tid; m < n_groups; m += kSelThreads) {
+        const uint32_t key = skey[m];
+        if (key != 0 && (key >> 21) == (uint32_t)fb) atomicAdd(&hist[(key >> 10) & 2047u], 1u);
+      }
+      int dg = 0, ab2 = 0;
+      locate_bin(hist + tid * (kStreamBins / kSelThreads), kStreamBins / kSelThreads, rho - ab, wsum, out2, dg, ab2);
+      floor_key = ((uint32_t)fb << 21) | ((uint32_t)dg << 10);
+    }
+  }
+  if (tid == 0) {
+    if (g.over) report(p.status, SPEC_ERR_BAD_ARG);
+    int32_t* hd = p.head + (int64_t)unit * p.head_words;
+    hd[0] = (int32_t)floor_key;
+    hd[1] = 0;
+    hd[2] = 0;
+    hd[3] = 0;
+  }
+}
+
+// ---------------------------------------------------------------- 2. the sweep -------
+
+// Where a sweeping CTA's work item (one chunk of one unit) lies and what it copies in bulk.
+struct SweepItem {
+  UnitGeom g;
+  int32_t* hd;
+  uint32_t floor_key;
+  int chunk_id, mis, X, x0, x1, n_steps, xa, total, bx0, bx1;
+  bool active, bulk;
+};
+
+__device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int64_t item) {
+  SweepItem t;
+  const int unit = (int)(item / p.chunks_max);
+  t.chunk_id = (int)(item % p.chunks_max);
+  t.g = unit_geom(p, unit);
+  t.hd = p.head + (int64_t)unit * p.head_words;
+  t.floor_key = (uint32_t)__ldg(t.hd);
+  t.mis = (int)((reinterpret_cast<uintptr_t>(t.g.src) >> 2) & 3u);
+  t.X = t.g.e + t.mis;                                     // x = position + mis: multiples of four are 16-byte boundaries
+  t.x0 = t.chunk_id * p.chunk;
+  t.x1 = min(t.x0 + p.chunk, t.X);
+  t.active = t.floor_key != kNoSelection && t.x1 > t.x0;
+  t.n_steps = t.active ? (t.x1 - t.x0 + 127) >> 7 : 0;
+  // staged: [x0 - 4, x0 + n_steps * 128 + 4); the 16-byte aligned interior of the unit comes by bulk copy
+  t.xa = t.x0 - 4;
+  t.total = t.n_steps * 128 + 8;
+  t.bx0 = max(t.xa, t.mis ? 4 : 0);
+  t.bx1 = min(t.xa + t.total, t.X & ~3);
+  t.bulk = t.active && t.bx1 > t.bx0;
+  if (!t.bulk) t.bx0 = t.bx1 = t.xa + t.total;
+  return t;
+}
+
+// One CTA per item.  Eight small CTAs share an SM, so that the bulk copies of some overlap the
+// pooling of others (a persistent, double-buffered variant with fewer resident warps was slower).
+__global__ void __launch_bounds__(kSweepThreads, 8) stream_sweep_kernel(const StreamParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  __shared__ int wsum[kSweepWarps];
+  __shared__ uint64_t mbar;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const SweepItem t = sweep_item(p, blockIdx.x);
+  if (!t.active) return;
+  float* raw = reinterpret_cast<float*>(smem_raw);
+  const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&mbar);
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (t.bulk) {
+      const uint32_t bytes = (uint32_t)(t.bx1 - t.bx0) * 4u;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"((uint32_t)__cvta_generic_to_shared(raw + (t.bx0 - t.xa))), "l"(t.g.src + (t.bx0 - t.mis)), "r"(bytes), "r"(bar_a)
+                   : "memory");
+    }
+  }
+  for (int i = tid; i < t.total; i += kSweepThreads) {
+    const int x = t.xa + i;
+    if (x >= t.bx0 && x < t.bx1) { i += ((t.bx1 - x - 1) / kSweepThreads) * kSweepThreads; continue; }   // the bulk-copied part
+    const int pp = x - t.mis;
+    raw[i] = (pp >= 0 && pp < t.g.e) ? __ldg(t.g.src + pp) : -INFINITY;
+  }
+  __syncthreads();                                         // the barrier is initialised; the edges are in place
+  if (t.bulk) {
+    uint32_t ok = 0;
+    for (uint32_t tries = 0; tries < (1u << 20) && !ok; ++tries)
+      asm volatile("{\n.reg .pred q;\nmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\nselp.u32 %0, 1, 0, q;\n}"
+                   : "=r"(ok) : "r"(bar_a) : "memory");
+    if (!ok) {                                             // the copy never landed: the unit is handed to the generic path
+      report(p.status, SPEC_ERR_TIMEOUT);
+      atomicExch(t.hd + 3, 1);
+    }
+  }
+  // ---- pooled maxima straight from shared memory, kept in registers; warp w owns steps w, w + 4, ...
+  // Only the chunks at either end of the unit hold slots that are not positions.
+  const float floor_f = key_to_float(t.floor_key);
+  const float4* base4 = reinterpret_cast<const float4*>(raw + 4);
+  const bool edge = t.x0 < t.mis || t.x0 + t.n_steps * 128 > t.X;
+  float pooled[kMaxStepsPerWarp][4];
+  int mine = 0;
+#pragma unroll
+  for (int k = 0; k < kMaxStepsPerWarp; ++k) {
+    const int st = warp + k * kSweepWarps;
+    if (st < t.n_steps) {
+      const float4* at = base4 + st * 32 + lane;
+      const float4 pv = at[-1], cv = at[0], nv = at[1];
+      const float x[10] = {pv.y, pv.z, pv.w, cv.x, cv.y, cv.z, cv.w, nv.x, nv.y, nv.z};
+      float t3[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t3[i] = fmax3(x[i], x[i + 1], x[i + 2]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) pooled[k][u] = fmax3(t3[u], t3[u + 3], x[u + 6]);
+      if (edge) {
+        const int pp0 = t.x0 + st * 128 + lane * 4 - t.mis;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (pp0 + u < 0 || pp0 + u >= t.g.e) pooled[k][u] = __uint_as_float(0xFFFFFFFFu);   // not a position: never a candidate
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) mine += !(pooled[k][u] < floor_f) && __float_as_uint(pooled[k][u]) != 0xFFFFFFFFu;
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) pooled[k][u] = __uint_as_float(0xFFFFFFFFu);
+    }
+  }
+  // ---- my candidates go to my own segment of the unit's array, their number to the unit's header
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) wsum[warp] = incl;
+  __syncthreads();
+  int before = incl - mine, n_cta = 0;
+#pragma unroll
+  for (int w = 0; w < kSweepWarps; ++w) {
+    const int c = wsum[w];
+    if (w < warp) before += c;
+    n_cta += c;
+  }
+  if (tid == 0) t.hd[4 + t.chunk_id] = n_cta;              // a segment is as long as the chunk: it cannot overflow
+  if (mine == 0) return;
+  uint2* dst = p.cand + t.g.cand_off + (int64_t)t.chunk_id * p.chunk + before;
+#pragma unroll
+  for (int k = 0; k < kMaxStepsPerWarp; ++k) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float v = pooled[k][u];
+      if (!(v < floor_f) && __float_as_uint(v) != 0xFFFFFFFFu)
+        *dst++ = make_uint2(to_key(v), (uint32_t)(t.x0 + (warp + k * kSweepWarps) * 128 + lane * 4 + u - t.mis));
+    }
+  }
+}
+
+// ------------------------------------------------------------- 3. the finishing CTA --
+
+// Shared memory of stream_finish_kernel: radix histogram, the candidates, two position bitmaps
+// (or, instead of the bitmaps, the scratch of the generic selection).
+__host__ __device__ inline size_t stream_finish_bytes(int bitmap_words, int held_cap) {
+  const size_t maps = (size_t)bitmap_words * 8, generic = (size_t)(kSelWarps * 256 + 2 * kSelWarps + 8) * 4;
+  return (size_t)kStreamBins * 4 + (size_t)held_cap * 8 + (maps > generic ? maps : generic);
+}
+
+__global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const StreamParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  __shared__ int wsum[32];
+  __shared__ int out2[4];
+  __shared__ uint64_t mbar;
+  const int tid = threadIdx.x;
+  const int unit = blockIdx.x;
+  const UnitGeom g = unit_geom(p, unit);
+  const int32_t* hd = p.head + (int64_t)unit * p.head_words;
+  uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);
+  uint2* held = reinterpret_cast<uint2*>(hist + kStreamBins);
+  uint32_t* map_gt = reinterpret_cast<uint32_t*>(held + p.held_cap);
+  uint32_t* map_eq = map_gt + p.bitmap_words;
+  const bool any_selects = (g.take[0] > 0 && g.take[0] < g.e) || (p.n_vert > 0 && g.take[1] > 0 && g.take[1] < g.e);
+  // ---- gather the candidates of the unit's chunks
+  int n_cand = 0, n_real = 0;                              // slots gathered (padding pairs included), real candidates
+  bool failed = hd[3] != 0;
+  if (any_selects) {
+    const int mis = (int)((reinterpret_cast<uintptr_t>(g.src) >> 2) & 3u);
+    const int n_chunks = (g.e + mis + p.chunk - 1) / p.chunk;          // <= kSelThreads, checked on the host
+    const uint2* segs = p.cand + g.cand_off;
+    const int raw_cnt = tid < n_chunks ? hd[4 + tid] : 0;
+    const int my_cnt = (raw_cnt + 1) & ~1;                 // rounded up to a whole 16 bytes
+    int total;
+    const int mine_at = block_exclusive_scan(my_cnt, wsum, total);
+    __syncthreads();
+    block_exclusive_scan(raw_cnt, wsum, n_real);
+    failed = failed || total > p.held_cap;
+    if (!failed) {
+      // One bulk asynchronous copy per chunk, all in flight together.  Bulk copies move multiples of
+      // 16 bytes to 16-byte aligned places, so every chunk's candidates start at an even slot and
+      // an odd count drags one stale pair along, marked as padding afterwards.
+      const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&mbar);
+      if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"((uint32_t)total * 8u) : "memory");
+      }
+      __syncthreads();
+      if (my_cnt > 0) {
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"((uint32_t)__cvta_generic_to_shared(held + mine_at)), "l"(segs + (int64_t)tid * p.chunk),
+                       "r"((uint32_t)my_cnt * 8u), "r"(bar_a) : "memory");
+      }
+      uint32_t ok = total == 0;
+      for (uint32_t tries = 0; tries < (1u << 20) && !ok; ++tries)
+        asm volatile("{\n.reg .pred q;\nmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\nselp.u32 %0, 1, 0, q;\n}"
+                     : "=r"(ok) : "r"(bar_a) : "memory");
+      if (__syncthreads_or(!ok)) {                         // the copies never landed: the generic path serves the unit
+        if (tid == 0) report(p.status, SPEC_ERR_TIMEOUT);
+        failed = true;
+      } else {
+        if (raw_cnt & 1) held[mine_at + raw_cnt] = make_uint2(0u, kNoSelection);   // padding pair
+        n_cand = total;
+      }
+    }
+  }
+  const uint2* cand = held;
+  const int n_budgets = p.n_vert > 0 ? 2 : 1;
+  for (int b = 0; b < n_budgets; ++b) {
+    int32_t* idx = b == 0 ? p.idx_out + (int64_t)unit * p.c_max : p.vert_out + (int64_t)unit * p.n_vert;
+    int32_t* cnt = b == 0 ? p.count_out : p.vert_count_out;
+    const int width = b == 0 ? p.c_max : p.n_vert;
+    const int tail = b == 0 ? g.forced : 0;
+    const int tk = g.take[b];
+    __syncthreads();
+    if (tk > 0 && tk < g.e) {
+      if (failed || n_real < tk) {
+        __syncthreads();
+        // generic selection: pooled keys recomputed from global memory in every pass
+        SelectScratch sc;
+        sc.hist = map_gt;
+        sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
+        KeySource key;
+        key.scores = g.src;
+        key.e = g.e; key.pool = SPEC_POOL_MAX; key.k = 7;
+        key.keys = nullptr;
+        uint32_t T;
+        int need_eq;
+        radix_select(key, g.e, tk, sc, T, need_eq);
+        ordered_emit(key, g.e, T, need_eq, sc, [&](int rank, int j) { idx[rank] = j; });
+      } else {
+        // ---- exact threshold among the candidates
+        uint32_t prefix = 0, mask = 0;
+        int remaining = tk;
+        for (int pass = 0; pass < 3; ++pass) {
+          const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
+          const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+          for (int i = tid; i < kStreamBins; i += kSelThreads) hist[i] = 0;
+          __syncthreads();
+          for (int i0 = 0; i0 < n_cand; i0 += kSelThreads) {
+            // lanes of a warp with the same digit add once: the candidates share their leading bits
+            const int i = i0 + tid;
+            const uint2 ck = i < n_cand ? cand[i] : make_uint2(0u, kNoSelection);
+            const uint32_t kk = ck.x;
+            const bool in = ck.y != kNoSelection && (kk & mask) == prefix;
+            const uint32_t dgt = (kk >> shift) & dmask;
+            if (pass == 0) {
+              const uint32_t act = __ballot_sync(0xffffffffu, in);
+              if (in) {
+                const uint32_t same = __match_any_sync(act, dgt);
+                if ((tid & 31) == __ffs(same) - 1) atomicAdd(&hist[dgt], (uint32_t)__popc(same));
+              }
+            } else if (in) {
+              atomicAdd(&hist[dgt], 1u);
+            }
+          }
+          int dg = 0, ab = 0;
+          locate_bin(hist + tid * (kStreamBins / kSelThreads), kStreamBins / kSelThreads, remaining, wsum, out2, dg, ab);
+          remaining -= ab;
+          prefix |= (uint32_t)dg << shift;
+          mask |= dmask << shift;
+        }
+        const uint32_t T = prefix;
+        const int need_eq = remaining;
+        // ---- winners and ties into position bitmaps, then out in ascending position
+        const int n_words = (g.e + 31) >> 5;
+        for (int w = tid; w < n_words; w += kSelThreads) { map_gt[w] = 0; map_eq[w] = 0; }
+        __syncthreads();
+        for (int i = tid; i < n_cand; i += kSelThreads) {
+          const uint2 c = cand[i];
+          if (c.y == kNoSelection) continue;
+          if (c.x > T) atomicOr(&map_gt[c.y >> 5], 1u << (c.y & 31));
+          else if (c.x == T) atomicOr(&map_eq[c.y >> 5], 1u << (c.y & 31));
+        }
+        __syncthreads();
+        // Output rank of a position = winners (and ties) before it: an exclusive count per group of
+        // a few words, kept where the histogram was, plus the words of its own group up to its bit.
+        const int gw = (n_words + 2 * kSelThreads - 1) / (2 * kSelThreads);   // words per group, two groups per thread
+        int* grp_gt = reinterpret_cast<int*>(hist);
+        int* grp_eq = grp_gt + 2 * kSelThreads;
+        int gt0 = 0, eq0 = 0, gt1 = 0, eq1 = 0;
+        for (int w = 2 * tid * gw; w < min((2 * tid + 1) * gw, n_words); ++w) { gt0 += __popc(map_gt[w]); eq0 += __popc(map_eq[w]); }
+        for (int w = (2 * tid + 1) * gw; w < min((2 * tid + 2) * gw, n_words); ++w) { gt1 += __popc(map_gt[w]); eq1 += __popc(map_eq[w]); }
+        int tot_gt, tot_eq;
+        const int sg = block_exclusive_scan(gt0 + gt1, wsum, tot_gt);
+        __syncthreads();
+        const int sq = block_exclusive_scan(eq0 + eq1, wsum, tot_eq);
+        grp_gt[2 * tid] = sg; grp_gt[2 * tid + 1] = sg + gt0;
+        grp_eq[2 * tid] = sq; grp_eq[2 * tid + 1] = sq + eq0;
+        __syncthreads();
+#pragma unroll 2
+        for (int i = tid; i < n_cand; i += kSelThreads) {
+          const uint2 c = cand[i];
+          if (c.x < T || c.y == kNoSelection) continue;
+          const int w = (int)(c.y >> 5), grp = w / gw;
+          const uint32_t below = (1u << (c.y & 31)) - 1u;
+          int g_before = grp_gt[grp] + __popc(map_gt[w] & below), q_before = grp_eq[grp] + __popc(map_eq[w] & below);
+          for (int ww = grp * gw; ww < w; ++ww) { g_before += __popc(map_gt[ww]); q_before += __popc(map_eq[ww]); }
+          if (c.x > T) idx[g_before + min(q_before, need_eq)] = (int32_t)c.y;
+          else if (q_before < need_eq) idx[g_before + q_before] = (int32_t)c.y;
+        }
+      }
+    } else {
+      for (int q = tid; q < tk; q += kSelThreads) idx[q] = q;        // every eligible position is kept
+    }
+    for (int q = tk + tid; q < width; q += kSelThreads) idx[q] = (q - tk < tail) ? g.e + (q - tk) : -1;
+    if (cnt && tid == 0) cnt[unit] = tk + tail;
+  }
+}
+
+// ------------------------------------------------------------------ host side ---------
+
+int run_stream_topk(const spec_problem* pr, const float* scores, int c_max, int n_forced_tail, int32_t* idx_out,
+                    int32_t* count_out, int n_vert, int32_t* vert_out, int32_t* vert_count_out, void* workspace,
+                    size_t workspace_bytes, int32_t* status_word, cudaStream_t st, bool* done) {
+  *done = false;
+  if (!workspace) return SPEC_OK;
+  const WorkspacePlan wp = plan_workspace(pr);
+  if (workspace_bytes < wp.total) return SPEC_OK;
+  const int max_len = max_seq_len(pr);
+  if (max_len < 1) return SPEC_OK;
+  const int64_t n_units = (int64_t)pr->n_seq * pr->n_layers * pr->n_kv_heads;
+
+  StreamParams p = {};
+  p.scores = scores; p.cu = pr->cu_seqlens; p.T = pr->total_tokens; p.n_in = pr->n_in;
+  p.L = pr->n_layers; p.H = pr->n_kv_heads; p.n_forced = n_forced_tail; p.c_max = c_max; p.n_vert = n_vert;
+  // chunks of 4096 positions (a warp keeps its 8 steps of pooled values in registers), smaller
+  // while that leaves SMs without a CTA
+  int chunk = kSelChunkMax;
+  static_assert(kSelChunkMax == kMaxStepsPerWarp * kSweepWarps * 128, "a sweeping warp keeps its steps in registers");
+  while (chunk > kSelChunkMin && n_units * (((int64_t)max_len + 3 + chunk - 1) / chunk) < 1184) chunk >>= 1;
+  p.chunk = chunk;
+  p.chunks_max = (int)(((int64_t)max_len + 3 + chunk - 1) / chunk);
+  if (p.chunks_max > kSelThreads) return SPEC_OK;          // the finishing CTA reads one segment count per thread
+  p.bitmap_words = ((max_len + 31) / 32 + 3) & ~3;
+  p.max_len = max_len;
+  const size_t smem_sweep = (size_t)(chunk + 8 + 128) * 4;
+  // the floor lets through about 1.6 to 2.5 times the budget (less for larger budgets)
+  p.held_cap = (3 * std::max(c_max, n_vert) + 2048 + 3) & ~3;
+  if (stream_finish_bytes(p.bitmap_words, p.held_cap) > (size_t)kSmemLimit - 1024) {
+    // a large budget: what fits (the floor lets through about 1.6 times a budget of thousands)
+    const int64_t room = ((int64_t)kSmemLimit - 1024 - (int64_t)stream_finish_bytes(p.bitmap_words, 0)) / 8;
+    if (room < 2 * (int64_t)std::max(c_max, n_vert) + 2048) return SPEC_OK;   // too long or too large a budget for the finishing CTA
+    p.held_cap = (int)(room & ~(int64_t)3);
+  }
+  const size_t smem_finish = stream_finish_bytes(p.bitmap_words, p.held_cap);
+  if (n_units * p.chunks_max > 0x7fffffffLL) return SPEC_OK;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  p.head = reinterpret_cast<int32_t*>(ws + wp.sel_head_off);
+  p.head_words = wp.sel_head_words;
+  p.cand = reinterpret_cast<uint2*>(ws + wp.sel_cand_off);
+  p.row_entries = wp.sel_row_entries;
+  p.idx_out = idx_out; p.count_out = count_out; p.vert_out = vert_out; p.vert_count_out = vert_count_out;
+  p.status = status_word;
+
+  static int set[64] = {0};
+  int dev = 0;
+  SPEC_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SPEC_OK;
+  if (!__atomic_load_n(&set[dev], __ATOMIC_ACQUIRE)) {
+    SPEC_CUDA_OK(cudaFuncSetAttribute(stream_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - 1024));
+    __atomic_store_n(&set[dev], 1, __ATOMIC_RELEASE);
+  }
+  sample_floor_kernel<<<(unsigned)n_units, kSelThreads, 0, st>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  stream_sweep_kernel<<<(unsigned)(n_units * p.chunks_max), kSweepThreads, smem_sweep, st>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  stream_finish_kernel<<<(unsigned)n_units, kSelThreads, smem_finish, st>>>(p);
+  SPEC_CUDA_OK(cudaGetLastError());
+  *done = true;
+  return SPEC_OK;
+}
+
+}  // namespace spec

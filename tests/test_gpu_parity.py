@@ -189,29 +189,36 @@ def test_score_wide_gqa_group_in_five_row_groups(B, W, oracle):
 # ------------------------------------------------------------------ selection ---------
 
 def run_topk_case(B, W, oracle, scores, cu, pool, k, c_max, forced, exact=True):
+    """spec_pool_topk on given scores against the oracle, twice: without a workspace (the selection that keeps
+    a unit resident in a thread-block cluster) and with one (the streaming selection, where it applies)."""
     L, H, T = scores.shape
     cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda") if len(cu) > 2 else None   # must outlive the call
     pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=128, n_lookahead=1, n_window=0,
                         softmax_scale=1.0, total_tokens=T, n_in=int(max(np.diff(cu))), n_seq=len(cu) - 1,
                         cu_seqlens=cu_t)
-    idx = torch.full((len(cu) - 1, L, H, c_max), -7, dtype=torch.int32, device="cuda")
-    cnt = torch.full((len(cu) - 1, L, H), -7, dtype=torch.int32, device="cuda")
-    B.spec_pool_topk(pr, torch.from_numpy(scores).cuda(), pool, k, c_max, forced, idx, cnt)
-    torch.cuda.synchronize()
     oidx, ocnt, pooled, th = oracle.pool_topk(scores.astype(np.float64), cu, pool, k, c_max, forced)
-    np.testing.assert_array_equal(cnt.cpu().numpy(), ocnt)
-    if exact:
-        np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
-    else:
-        gi = idx.cpu().numpy()
-        for s in range(len(cu) - 1):
-            for l in range(L):
-                for h in range(H):
-                    nf = min(forced, cu[s + 1] - cu[s])
-                    e = cu[s + 1] - cu[s] - nf
-                    ge, oe = gi[s, l, h], oidx[s, l, h]
-                    assert_index_sets_match(ge[(ge >= 0) & (ge < e)], oe[(oe >= 0) & (oe < e)],
-                                            pooled[l, h, cu[s]:cu[s + 1]], th[s, l, h])
+    scores_t = torch.from_numpy(scores).cuda()
+    ws = torch.empty(max(B.spec_workspace_bytes(pr), 16), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for workspace in (None, ws):
+        idx = torch.full((len(cu) - 1, L, H, c_max), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((len(cu) - 1, L, H), -7, dtype=torch.int32, device="cuda")
+        B.spec_pool_topk(pr, scores_t, pool, k, c_max, forced, idx, cnt, workspace=workspace, status_word=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        np.testing.assert_array_equal(cnt.cpu().numpy(), ocnt)
+        if exact:
+            np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
+        else:
+            gi = idx.cpu().numpy()
+            for s in range(len(cu) - 1):
+                for l in range(L):
+                    for h in range(H):
+                        nf = min(forced, cu[s + 1] - cu[s])
+                        e = cu[s + 1] - cu[s] - nf
+                        ge, oe = gi[s, l, h], oidx[s, l, h]
+                        assert_index_sets_match(ge[(ge >= 0) & (ge < e)], oe[(oe >= 0) & (oe < e)],
+                                                pooled[l, h, cu[s]:cu[s + 1]], th[s, l, h])
 
 
 def test_topk_exact_with_ties_runs_and_forced_tail(B, W, oracle):
@@ -558,22 +565,144 @@ def test_specpc_config3_full(B, W, oracle):
 
 # ------------------------------------------------------------------ widening rows -----
 
-def test_vertical_indices_are_a_second_top_k(B, W, oracle):
-    """Algorithm 1 line 11: i_vert = topk(s, n_vert) on the same pooled scores as i_cache (line 13) is the
-    same call with another budget; the smaller set is contained in the larger one."""
-    w = small(W, n_in=5000, c_max=256)
-    g = Gpu(B, W, w, [0, 1])
-    scores = g.score()
-    sc = scores.cpu().numpy().astype(np.float64)
-    i_cache, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 256, forced=w.n_window)
-    i_vert, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 1024)
-    o_vert, _, _, _ = oracle.pool_topk(sc, g.cu, oracle.POOL_MAX, w.pool_k, 1024)
-    np.testing.assert_array_equal(i_vert.cpu().numpy(), o_vert)
-    small_set, _ = g.topk(scores, B.POOL_MAX, w.pool_k, 256)
-    for l in range(2):
-        for h in range(w.n_kv_heads):
-            assert set(small_set[0, l, h].tolist()) <= set(i_vert[0, l, h].tolist())
-    assert i_cache.shape[-1] == 256
+def run_vert_case(B, oracle, scores, cu, k, c_max, forced, n_vert):
+    """spec_pool_topk_vert against two oracle selections on the same pooled scores."""
+    L, H, T = scores.shape
+    n_seq = len(cu) - 1
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda") if n_seq > 1 else None
+    pr = B.make_problem(n_layers=L, n_q_heads=H, n_kv_heads=H, head_dim=128, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=T, n_in=int(max(np.diff(cu))), n_seq=n_seq, cu_seqlens=cu_t)
+    s64 = scores.astype(np.float64)
+    o_cache, o_cnt, _, _ = oracle.pool_topk(s64, cu, oracle.POOL_MAX, k, c_max, forced)
+    # i_vert is the plain top-n_vert of the positions before the forced tail: the oracle gets them as
+    # sequences cut at the tail, with the same pooling clipped to that range
+    o_vert = np.full((n_seq, L, H, n_vert), -1, dtype=np.int32)
+    o_vcnt = np.zeros((n_seq, L, H), dtype=np.int32)
+    for s in range(n_seq):
+        n = cu[s + 1] - cu[s]
+        e = n - min(forced, n)
+        if e > 0:
+            oi, oc, _, _ = oracle.pool_topk(s64[:, :, cu[s]:cu[s] + e].copy(), [0, e], oracle.POOL_MAX, k, n_vert, 0)
+            o_vert[s], o_vcnt[s] = oi[0], oc[0]
+    ws = torch.empty(max(B.spec_workspace_bytes(pr), 16), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for workspace in (None, ws):                       # cluster-resident and streaming selection
+        idx = torch.full((n_seq, L, H, c_max), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((n_seq, L, H), -7, dtype=torch.int32, device="cuda")
+        vidx = torch.full((n_seq, L, H, n_vert), -7, dtype=torch.int32, device="cuda")
+        vcnt = torch.full((n_seq, L, H), -7, dtype=torch.int32, device="cuda")
+        B.spec_pool_topk_vert(pr, torch.from_numpy(scores).cuda(), B.POOL_MAX, k, c_max, forced, idx, cnt, n_vert, vidx, vcnt,
+                              workspace=workspace, status_word=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        np.testing.assert_array_equal(idx.cpu().numpy(), o_cache)
+        np.testing.assert_array_equal(cnt.cpu().numpy(), o_cnt)
+        np.testing.assert_array_equal(vidx.cpu().numpy(), o_vert)
+        np.testing.assert_array_equal(vcnt.cpu().numpy(), o_vcnt)
+
+
+def test_vertical_and_cache_indices_from_one_sweep(B, W, oracle):
+    """Algorithm 1 lines 11 and 13: i_vert = topk(s, n_vert) and i_cache = topk(s, C_max - n_window) + window
+    from the same pooled scores, in one call that reads the scores once."""
+    rng = np.random.default_rng(21)
+    x = rng.random((2, 2, 20000)).astype(np.float32) ** 6
+    run_vert_case(B, oracle, x, [0, 20000], 7, 256, 32, 2048)            # the paper's n_vert and window
+    run_vert_case(B, oracle, x, [0, 20000], 7, 2048, 0, 256)             # vertical budget below the cache budget
+    run_vert_case(B, oracle, x, [0, 20000], 7, 256, 32, 30000)           # n_vert beyond the sequence: all, -1 padded
+    ties = (rng.integers(0, 6, size=(1, 3, 9000)) / 4).astype(np.float32)  # long runs of equal pooled values
+    run_vert_case(B, oracle, ties, [0, 9000], 7, 300, 16, 1000)
+    run_vert_case(B, oracle, ties, [0, 2000, 2000, 2003, 9000], 5, 64, 8, 100)   # ragged, an empty and a tiny sequence
+    # from real scores of the scoring call, long enough for a cluster of several CTAs
+    w = small(W, n_in=40000, c_max=256)
+    g = Gpu(B, W, w, [0])
+    sc = g.score().cpu().numpy()
+    run_vert_case(B, oracle, sc, g.cu, w.pool_k, 256, w.n_window, 2048)
+
+
+STRUCTURED = {
+    "random": lambda rng, n: rng.random(n) ** 6,
+    "rising": lambda rng, n: np.linspace(0.0, 1.0, n),
+    "falling": lambda rng, n: np.linspace(1.0, 0.0, n),
+    "recency_decay": lambda rng, n: np.exp(-(n - 1 - np.arange(n)) / (n / 12.0)) * (0.5 + rng.random(n)),
+    "winners_in_one_sixteenth": lambda rng, n: np.where((np.arange(n) >= 5 * (n // 16)) & (np.arange(n) < 6 * (n // 16)),
+                                                         1.0 + rng.random(n), 0.01 * rng.random(n)),
+    "few_distinct_values": lambda rng, n: rng.integers(0, 5, n) / 8.0,
+}
+
+
+def test_topk_structured_score_vectors_exact_and_not_slow(B, W, oracle):
+    """Score vectors with the shapes real attention mass takes (recency-biased, trending, concentrated) and
+    large budgets, at the 128K unit size: exact lists, and no input shape may cost more than a small
+    multiple of random scores."""
+    rng = np.random.default_rng(31)
+    n, H = 131072, 8
+    pr = B.make_problem(n_layers=1, n_q_heads=H, n_kv_heads=H, head_dim=128, n_lookahead=1, n_window=0,
+                        softmax_scale=1.0, total_tokens=n, n_in=n)
+    ws = torch.empty(B.spec_workspace_bytes(pr), dtype=torch.uint8, device="cuda")
+    times = {}
+    for name, fn in STRUCTURED.items():
+        for c_max in (2048, 4096, 8192):
+            if name not in ("random", "recency_decay") and c_max != 2048:
+                continue
+            x = np.stack([fn(rng, n) for _ in range(H)])[None].astype(np.float32)
+            xt = torch.from_numpy(x).cuda()
+            idx = torch.full((1, 1, H, c_max), -7, dtype=torch.int32, device="cuda")
+            B.spec_pool_topk(pr, xt, B.POOL_MAX, 7, c_max, 0, idx, None, workspace=ws)
+            torch.cuda.synchronize()
+            oidx, _, _, _ = oracle.pool_topk(x.astype(np.float64), [0, n], oracle.POOL_MAX, 7, c_max, 0)
+            np.testing.assert_array_equal(idx.cpu().numpy(), oidx, err_msg="%s c_max=%d" % (name, c_max))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                B.spec_pool_topk(pr, xt, B.POOL_MAX, 7, c_max, 0, idx, None, workspace=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            times[(name, c_max)] = e0.elapsed_time(e1) / 10
+    print("select ms per call (8 units of 131072):", {"%s/%d" % k: round(v, 4) for k, v in times.items()})
+    base = times[("random", 2048)]
+    for key, t in times.items():
+        if key[0] == "few_distinct_values":        # thousands of positions tie at the threshold: the generic path, exact but slow
+            continue
+        assert t <= 3.0 * base + 0.02, "%s takes %.3f ms against %.3f ms for random scores" % (key, t, base)
+
+
+def test_topk_unit_too_long_for_a_cluster_takes_the_generic_path(B, W, oracle):
+    rng = np.random.default_rng(41)
+    n = 2_000_003
+    x = (rng.random((1, 1, n)) ** 4).astype(np.float32)
+    x[0, 0, ::50000] = 0.9                                           # ties at the top
+    run_topk_case(B, W, oracle, x, [0, n], 0, 7, 1000, 32)
+
+
+def test_selection_skips_a_sequence_longer_than_the_given_bound(B, W, oracle):
+    """With cu_seqlens the lengths live on the device and n_in is only the caller's bound.  A sequence longer
+    than the bound is reported and skipped: no write outside the shared memory sized from the bound."""
+    rng = np.random.default_rng(51)
+    cu = [0, 3000, 3100]
+    x = rng.random((1, 2, 3100)).astype(np.float32)
+    cu_t = torch.tensor(cu, dtype=torch.int32, device="cuda")
+    pr = B.make_problem(n_layers=1, n_q_heads=2, n_kv_heads=2, head_dim=64, n_lookahead=1, n_window=0, softmax_scale=1.0,
+                        total_tokens=3100, n_in=200, n_seq=2, cu_seqlens=cu_t)            # 200 < 3000: too small a bound
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    idx = torch.full((2, 1, 2, 16), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((2, 1, 2), -7, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.spec_workspace_bytes(pr), dtype=torch.uint8, device="cuda")
+    o, _, _, _ = oracle.pool_topk(x.astype(np.float64), cu, oracle.POOL_MAX, 7, 16, 0)
+    for workspace in (None, ws):                                                 # both selection paths
+        B.spec_pool_topk(pr, torch.from_numpy(x).cuda(), B.POOL_MAX, 7, 16, 0, idx, cnt, workspace=workspace, status_word=status)
+        torch.cuda.synchronize()
+        assert status.item() == B.ERR_BAD_ARG
+        assert cnt[0].tolist() == [[0, 0]] and cnt[1].tolist() == [[16, 16]]     # the short sequence is still served
+        np.testing.assert_array_equal(idx[1].cpu().numpy(), o[1])
+        assert (idx[0] == -1).all()
+        status.zero_()
+    keep = torch.full((2, 200), -7, dtype=torch.int32, device="cuda")
+    n_keep = torch.full((2,), -7, dtype=torch.int32, device="cuda")
+    B.specpc_token_select(pr, torch.from_numpy(x).cuda(), B.REDUCE_SUM, B.POOL_MAX, 7, 8, 2, 0, keep, 200, n_keep, ws,
+                          status_word=status)
+    torch.cuda.synchronize()
+    assert status.item() == B.ERR_BAD_ARG
+    assert n_keep[0].item() == 0 and 8 <= n_keep[1].item() <= 40
 
 
 def test_gather_tokens_bit_exact(B, W, oracle):

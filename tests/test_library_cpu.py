@@ -82,7 +82,11 @@ def test_bad_call_arguments_are_rejected_on_the_host(B):
     assert L.spec_pool_topk(ctypes.byref(pr), one, 2, 7, 16, 0, one, None, None, 0, None, None) == B.ERR_BAD_ARG
     assert L.specpc_token_select(ctypes.byref(pr), one, 1, 2, 7, 16, 8, 4, one, 19, one, one, 1 << 30,
                                  None, None) == B.ERR_BAD_ARG
-    assert L.specpc_token_select_static(ctypes.byref(pr), one, 1, 2, 7, 16, 8, 4, one, 1024, one, None, None) == B.ERR_BAD_ARG
+    # ... and the workspace-free variant has no room for its second vector: refused by name, before any launch
+    assert L.specpc_token_select_static(ctypes.byref(pr), one, 1, 2, 7, 16, 8, 4, one, 1024, one, None, None) == B.ERR_UNSUPPORTED
+    assert "SPEC_POOL_AVG_THEN_MAX" in B.spec_last_error()
+    assert L.spec_pool_topk_vert(ctypes.byref(pr), one, 0, 7, 16, 0, one, None, 0, one, None, None, 0, None, None) == B.ERR_BAD_ARG
+    assert L.spec_pool_topk_vert(ctypes.byref(pr), one, 0, 7, 16, 0, one, None, 8, None, None, None, 0, None, None) == B.ERR_BAD_ARG
     assert L.spec_score(ctypes.byref(pr), one, one, None, 0, 2, one, one, 1 << 30, None, None) == B.ERR_BAD_ARG
     # prompt compression
     assert L.spec_gather_tokens(ctypes.byref(pr), one, None, None, 16, one, one, None, 64, one, None, None) == B.ERR_BAD_ARG

@@ -43,7 +43,7 @@ class Gpu:
     def topk(self, scores, pool, pool_k, c_max, forced=0):
         idx = torch.full((self.w.n_seq, self.L, self.w.n_kv_heads, c_max), -7, dtype=torch.int32, device="cuda")
         cnt = torch.full((self.w.n_seq, self.L, self.w.n_kv_heads), -7, dtype=torch.int32, device="cuda")
-        self.B.spec_pool_topk(self.pr, scores, pool, pool_k, c_max, forced, idx, cnt, status_word=self.status)
+        self.B.spec_pool_topk(self.pr, scores, pool, pool_k, c_max, forced, idx, cnt, workspace=self.ws, status_word=self.status)
         torch.cuda.synchronize()
         assert self.status.item() == 0
         return idx, cnt
