@@ -770,6 +770,10 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
     return fail(SPEC_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", workspace_bytes, wp.total);
   rc = check_device();
   if (rc != SPEC_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the whole output is overwritten: tokens that no sequence covers read as 0, and pass 2 adds into it
+  const size_t out_bytes = (size_t)pr->n_layers * pr->n_kv_heads * (size_t)pr->total_tokens * sizeof(float);
+  if (out_bytes) SPEC_CUDA_OK(cudaMemsetAsync(scores_out, 0, out_bytes, st));
   const int64_t tokens = pr->cu_seqlens ? pr->total_tokens : pr->n_in;
   if (tokens == 0) return SPEC_OK;
 
@@ -815,13 +819,24 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
   p.a = (float)((double)pr->softmax_scale * 1.4426950408889634);
   p.stage_bytes = (uint32_t)kTileKeys * d * 2;
 
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int n_ctas = wp.score_ctas;
   const unsigned n_units = (unsigned)(pr->n_seq * pr->n_layers * pr->n_kv_heads);
   auto pass1 = score_kernel<1, false>;
   auto pass2 = reduce == SPEC_REDUCE_MAX ? score_kernel<2, true> : score_kernel<2, false>;
-  SPEC_CUDA_OK(cudaMemsetAsync(scores_out, 0, (size_t)pr->n_layers * pr->n_kv_heads * (size_t)pr->total_tokens * sizeof(float), st));
-  int smem_set = 0;
+  // The kernels may use all of an SM's shared memory; the attribute is set once per device (it is per
+  // function and context, so setting it per call would race between host threads).
+  {
+    static int set[64] = {0};
+    int dev = 0;
+    SPEC_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return fail(SPEC_ERR_UNSUPPORTED, "device ordinal %d is not supported", dev);
+    if (!__atomic_load_n(&set[dev], __ATOMIC_ACQUIRE)) {
+      SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      SPEC_CUDA_OK(cudaFuncSetAttribute(score_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      __atomic_store_n(&set[dev], 1, __ATOMIC_RELEASE);
+    }
+  }
   for (int g = 0; g < n_groups; ++g) {
     p.row0 = g * rows_group;
     p.M = std::min(rows_group, M - p.row0);
@@ -839,11 +854,6 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
     p.n_stages = stages;
     int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
     if (smem < 120 * 1024) smem = 120 * 1024;             // one CTA per SM: each CTA owns the whole TMEM
-    if (smem > smem_set) {
-      SPEC_CUDA_OK(cudaFuncSetAttribute(pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-      SPEC_CUDA_OK(cudaFuncSetAttribute(pass2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-      smem_set = smem;
-    }
     pass1<<<n_ctas, kThreads, smem, st>>>(tm_q, tm_k, p);
     SPEC_CUDA_OK(cudaGetLastError());
     merge_kernel<<<n_units, 128, 0, st>>>(p, n_ctas);

@@ -55,6 +55,9 @@ class Workload:
     sink_gain: float = 0.0          # >0: key 0 is planted with this gain
     n_neighbor: int = 0             # SpecPC neighbour radius
     page_size: int = 0              # >0: paged destination cache
+    l_skip: int = 0                 # SpecPC: draft layers left out of the token scores
+    paper_specpc: bool = False      # SpecPC run with the paper's own settings (max reductions, window row weights,
+                                    # average pool then max pool before the selection, window always kept)
 
     @property
     def rows(self) -> int:
@@ -88,6 +91,11 @@ CONFIGS: List[Workload] = [
     Workload(name="c4_ragged_16seq", seed=4, n_layers=32, n_q_heads=32, n_kv_heads=8, head_dim=128,
              n_seq=16, len_lo=4096, len_hi=65536, n_lookahead=64, n_window=32, pool_k=7, c_max=1024,
              zipf_bias=True, page_size=16),
+    # not one of the five benchmark workloads: the SpecPC column of the paper's hyper-parameter table on the
+    # draft shape of workload 3 (n_window 64, n_lookahead 1, Pool Avg k = 64, n_neighbor 64, l_skip 8, C_max 1024)
+    Workload(name="c5_specpc_paper_settings", seed=5, n_layers=16, n_q_heads=32, n_kv_heads=8, head_dim=64,
+             n_in=32768, n_lookahead=1, n_window=64, pool_k=64, c_max=1024, planted="token",
+             n_planted=64, n_neighbor=64, l_skip=8, paper_specpc=True),
 ]
 
 

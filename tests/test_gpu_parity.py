@@ -461,7 +461,8 @@ def test_pipeline_config2_full_size_sampled_units(B, W, oracle):
 
 def test_pipeline_config4_ragged_paged_sampled_units(B, W, oracle):
     w = W.CONFIGS[4]
-    check_pipeline(B, W, oracle, w, [0, 1], units=[(0, 2), (1, 7)])
+    # layers spread over the model (first, middle, last), one sampled KV head of each
+    check_pipeline(B, W, oracle, w, [0, 15, 31], units=[(0, 2), (1, 7), (2, 4)])
 
 
 # ------------------------------------------------------------------ SpecPC ------------
@@ -561,6 +562,55 @@ def test_specpc_config3_full(B, W, oracle):
     near = np.flatnonzero(np.abs(tok - th[0]) <= band)
     for j in set(got) ^ ref_keep:
         assert np.any(np.abs(near - j) <= w.n_neighbor), "keep-list difference at %d outside the band" % j
+
+
+def test_specpc_paper_settings_from_real_scores(B, W, oracle):
+    """Algorithm 2 at the hyper-parameter table's SpecPC column, from the scoring call's own output on a
+    draft-shaped problem: max reduction over query rows, window rows weighted j / n_window, the first l_skip = 8
+    layers skipped by pointer offset, max over layers and heads, AvgPool(k) then MaxPool(n_neighbor) before the
+    selection, the window always kept.  Lists equal the oracle's except for positions whose pooled value lies
+    within the score tolerance of the threshold."""
+    n_window, l_skip, c_max = 64, 8, 1024
+    w = W.CONFIGS[3].replace(n_in=12000, n_layers=12, n_lookahead=1, n_window=n_window, n_planted=32, seed=17)
+    g = Gpu(B, W, w, list(range(w.n_layers)))
+    rw = torch.cat([torch.arange(1, n_window + 1, dtype=torch.float32) / n_window, torch.ones(w.n_lookahead)])
+    scores = g.score(reduce=B.REDUCE_MAX, row_weight=rw.cuda())
+    ref = oracle.spec_score(bits(g.q), bits(g.k), g.cu, w.n_lookahead, w.n_window, w.scale,
+                            row_weight=rw.double().numpy(), mode=oracle.MAX)
+    assert_scores_close(scores.cpu().numpy(), ref, g.cu)
+    used = scores[l_skip:]                                       # a view: the call sees layers l_skip.. only
+    pr = B.make_problem(n_layers=w.n_layers - l_skip, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                        n_lookahead=w.n_lookahead, n_window=w.n_window, softmax_scale=w.scale, total_tokens=w.n_in, n_in=w.n_in)
+    cap = c_max + n_window
+    for k, nb in ((64, 64), (32, 32)):
+        keep, n_keep = run_keep(B, pr, used, B.REDUCE_MAX, B.POOL_AVG_THEN_MAX, k, c_max, nb, n_window, cap, 1)
+        okeep, on, pooled, th = oracle.specpc_select(ref[l_skip:], g.cu, oracle.MAX, oracle.POOL_AVG_THEN_MAX, k, c_max, nb,
+                                                     n_window, cap)
+        assert n_keep[0] == on[0] == c_max + n_window            # exactly C_max tokens plus the window
+        got, want = keep[0, :n_keep[0]], okeep[0, :on[0]]
+        assert np.all(np.diff(got) > 0)
+        np.testing.assert_array_equal(got[-n_window:], np.arange(w.n_in - n_window, w.n_in))
+        band = 2e-3 * abs(th[0]) + 1e-6
+        for j in np.setxor1d(got, want):
+            assert abs(pooled[j] - th[0]) <= band, "k=%d: position %d decided outside the tolerance band" % (k, j)
+    # the single-stage average pool of Algorithm 1 line 10 as printed, on the same real scores
+    sc = scores.cpu().numpy()[:2]
+    run_topk_case(B, W, oracle, sc, g.cu, oracle.POOL_AVG, 7, 512, n_window, exact=False)
+    run_topk_case(B, W, oracle, sc, g.cu, oracle.POOL_AVG, 64, 512, 0, exact=False)
+    run_topk_case(B, W, oracle, sc, g.cu, oracle.POOL_MAX, 32, 512, 0)
+
+
+def test_score_zero_length_prompt_clears_the_output(B, W):
+    """n_in = 0 with a non-empty token axis: nothing to score, and the whole output buffer reads as zero."""
+    pr = B.make_problem(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_lookahead=2, n_window=2, softmax_scale=0.125,
+                        total_tokens=300, n_in=0)
+    q = torch.randn(1, 2, 4, 4, 64, device="cuda").to(torch.bfloat16)
+    k = torch.randn(2, 2, 300, 64, device="cuda").to(torch.bfloat16)
+    out = torch.full((2, 2, 300), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(B.spec_workspace_bytes(pr), 16), dtype=torch.uint8, device="cuda")
+    B.spec_score(pr, q, k, out, ws)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(out).item() == 0
 
 
 # ------------------------------------------------------------------ widening rows -----

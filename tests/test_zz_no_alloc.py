@@ -1,8 +1,10 @@
 """The workspace-free SpecPC entry point, for callers that cannot allocate device memory (for
 example code running inside a serving engine whose pool already owns the GPU): its scratch is an
-array inside the library.  It must give exactly what the workspace-taking entry point gives, on
-consecutive calls that reuse (and must not depend on) the array's old contents.  Collected last
-on purpose, so that a failure here cannot hide any other test."""
+array inside the library.  It must give exactly what the workspace-taking entry point gives, and
+what the CPU oracle gives, on consecutive calls that reuse (and must not depend on) the array's
+old contents.  Scores sit on a dyadic grid, so that fp32 sums and power-of-two averages are exact
+and the lists must be identical.  Collected last on purpose, so that a failure here cannot hide
+any other test."""
 import ctypes
 
 import numpy as np
@@ -36,25 +38,37 @@ def _both(B, pr, scores, n_seq, cap, args):
     return outs
 
 
-def test_static_scratch_entry_point_matches_workspace_entry_point_twice():
+def _oracle_keep(oracle, scores, cu, cap, args):
+    reduce, pool, k, c_max, nb, forced = args
+    keep, n_keep, _, _ = oracle.specpc_select(scores.astype(np.float64), cu, reduce, pool, k, c_max, nb, forced, cap)
+    return keep, n_keep
+
+
+def test_static_scratch_entry_point_matches_workspace_entry_point_and_oracle_twice(oracle):
     from paper_2506_08373_b200 import binding as B
     B.lib()
     rng = np.random.default_rng(77)
     # first call: long packed axis, so the array is left full of large token scores
     cu1, L1, H1 = [0, 3000, 3007, 9000], 4, 2
-    s1 = torch.from_numpy((rng.random((L1, H1, 9000)) ** 4 + 5.0).astype(np.float32)).cuda()
-    (k_ws, n_ws), (k_st, n_st) = _both(B, _problem(B, cu1, L1, H1), s1, 3, 5993,
-                                       (B.REDUCE_SUM, B.POOL_MAX, 7, 256, 8, 0))
-    np.testing.assert_array_equal(n_st, n_ws)
-    np.testing.assert_array_equal(k_st, k_ws)
-    assert n_ws.min() > 0
+    s1 = (rng.integers(0, 256, size=(L1, H1, 9000)) / 32 + 5.0).astype(np.float32)
+    args1 = (B.REDUCE_SUM, B.POOL_MAX, 7, 256, 8, 0)
+    (k_ws, n_ws), (k_st, n_st) = _both(B, _problem(B, cu1, L1, H1), torch.from_numpy(s1).cuda(), 3, 5993, args1)
+    k_or, n_or = _oracle_keep(oracle, s1, cu1, 5993, args1)
+    np.testing.assert_array_equal(n_st, n_or)
+    np.testing.assert_array_equal(k_st, k_or)
+    np.testing.assert_array_equal(n_ws, n_or)
+    np.testing.assert_array_equal(k_ws, k_or)
+    assert n_or.min() > 0
     # second call, right after: other shapes, smaller scores, other options; stale contents must not matter
     cu2, L2, H2 = [0, 500, 2100], 3, 4
-    s2 = torch.from_numpy((rng.random((L2, H2, 2100)) ** 2).astype(np.float32)).cuda()
-    (k_ws, n_ws), (k_st, n_st) = _both(B, _problem(B, cu2, L2, H2), s2, 2, 1600,
-                                       (B.REDUCE_MAX, B.POOL_AVG, 5, 100, 3, 16))
-    np.testing.assert_array_equal(n_st, n_ws)
-    np.testing.assert_array_equal(k_st, k_ws)
+    s2 = (rng.integers(0, 64, size=(L2, H2, 2100)) / 64).astype(np.float32)
+    args2 = (B.REDUCE_MAX, B.POOL_AVG, 4, 100, 3, 16)
+    (k_ws, n_ws), (k_st, n_st) = _both(B, _problem(B, cu2, L2, H2), torch.from_numpy(s2).cuda(), 2, 1600, args2)
+    k_or, n_or = _oracle_keep(oracle, s2, cu2, 1600, args2)
+    np.testing.assert_array_equal(n_st, n_or)
+    np.testing.assert_array_equal(k_st, k_or)
+    np.testing.assert_array_equal(n_ws, n_or)
+    np.testing.assert_array_equal(k_ws, k_or)
 
 
 def test_static_scratch_entry_point_rejects_more_tokens_than_its_array():
