@@ -44,7 +44,7 @@ SPEC_HIDDEN WorkspacePlan plan_workspace(const spec_problem* p);
 // Streaming selection: every chunk of a sequence owns a segment of the candidate array as long as
 // the chunk itself (at most kSelChunkMax positions, at least kSelChunkMin), so a sequence needs
 // its length plus a partial chunk; the chunks' candidate counts sit in the unit's header.
-constexpr int kSelChunkMax = 4096;
+constexpr int kSelChunkMax = 2048;
 constexpr int kSelChunkMin = 1024;
 constexpr int kSelCandSlack = 2 * kSelChunkMax;
 

@@ -28,7 +28,7 @@
 namespace spec {
 
 constexpr int kStreamBins = 2048;
-constexpr int kSweepThreads = 128;
+constexpr int kSweepThreads = 64;
 constexpr int kSweepWarps = kSweepThreads / 32;
 constexpr int kMaxStepsPerWarp = 8;              // 128-position steps a sweeping warp keeps in registers
 constexpr int kMaxSamples = 4096;
@@ -178,12 +178,12 @@ __device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int64_t i
   t.chunk_id = (int)(item % p.chunks_max);
   t.g = unit_geom(p, unit);
   t.hd = p.head + (int64_t)unit * p.head_words;
-  t.floor_key = (uint32_t)__ldg(t.hd);
+  t.floor_key = 0;                                         // read by the caller once the copy is under way
   t.mis = (int)((reinterpret_cast<uintptr_t>(t.g.src) >> 2) & 3u);
   t.X = t.g.e + t.mis;                                     // x = position + mis: multiples of four are 16-byte boundaries
   t.x0 = t.chunk_id * p.chunk;
   t.x1 = min(t.x0 + p.chunk, t.X);
-  t.active = t.floor_key != kNoSelection && t.x1 > t.x0;
+  t.active = t.x1 > t.x0;
   t.n_steps = t.active ? (t.x1 - t.x0 + 127) >> 7 : 0;
   // staged: [x0 - 4, x0 + n_steps * 128 + 4); the 16-byte aligned interior of the unit comes by bulk copy
   t.xa = t.x0 - 4;
@@ -197,13 +197,13 @@ __device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int64_t i
 
 // One CTA per item.  Eight small CTAs share an SM, so that the bulk copies of some overlap the
 // pooling of others (a persistent, double-buffered variant with fewer resident warps was slower).
-__global__ void __launch_bounds__(kSweepThreads, 8) stream_sweep_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(kSweepThreads, 16) stream_sweep_kernel(const StreamParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __shared__ int wsum[kSweepWarps];
   __shared__ uint64_t mbar;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const SweepItem t = sweep_item(p, blockIdx.x);
+  SweepItem t = sweep_item(p, blockIdx.x);
   if (!t.active) return;
   float* raw = reinterpret_cast<float*>(smem_raw);
   const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&mbar);
@@ -224,6 +224,9 @@ __global__ void __launch_bounds__(kSweepThreads, 8) stream_sweep_kernel(const St
     const int pp = x - t.mis;
     raw[i] = (pp >= 0 && pp < t.g.e) ? __ldg(t.g.src + pp) : -INFINITY;
   }
+  // The floor is fetched while the copy is in flight.  A unit that keeps everything or nothing needs no sweep,
+  // but its copy is awaited all the same: shared memory must not be given up with a copy under way.
+  t.floor_key = (uint32_t)__ldg(t.hd);
   __syncthreads();                                         // the barrier is initialised; the edges are in place
   if (t.bulk) {
     uint32_t ok = 0;
@@ -235,7 +238,8 @@ __global__ void __launch_bounds__(kSweepThreads, 8) stream_sweep_kernel(const St
       atomicExch(t.hd + 3, 1);
     }
   }
-  // ---- pooled maxima straight from shared memory, kept in registers; warp w owns steps w, w + 4, ...
+  if (t.floor_key == kNoSelection) return;
+  // ---- pooled maxima straight from shared memory, kept in registers; warp w owns steps w, w + 2, ...
   // Only the chunks at either end of the unit hold slots that are not positions.
   const float floor_f = key_to_float(t.floor_key);
   const float4* base4 = reinterpret_cast<const float4*>(raw + 4);
