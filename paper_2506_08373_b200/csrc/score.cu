@@ -10,23 +10,26 @@
 //            p = exp2(scale*log2e*S - c_i), reduced over columns thread-locally, one reduction per key
 //            and warpgroup.
 // Both passes are persistent, warp-specialised kernels: warp 0 feeds K tiles (and the unit's Q)
-// with TMA into a shared-memory ring, one (pass 1) or two (pass 2) threads issue tcgen05.mma into
-// TMEM, and four epilogue warpgroups (16 warps, four per SM sub-partition) drain the
-// accumulators with tcgen05.ld and do the exponentials.
-//   pass 1: work items of 128 rows x 256 keys (two ring stages as one N = 256 operand), two
-//           256-column buffers, all 16 epilogue warps on the same buffer (64 columns each);
-//   pass 2: 128 keys x 128 rows, four 128-column buffers; the warpgroups form two pairs, each
-//           with its own issuing thread and two buffers, the pair's warpgroups split a
-//           buffer's columns in halves.
+// with TMA into a shared-memory ring, two threads issue tcgen05.mma into TMEM, and four epilogue
+// warpgroups (16 warps, four per SM sub-partition) drain the accumulators with tcgen05.ld and
+// do the exponentials.  Every warpgroup owns one 128-column TMEM buffer.  A work item is
+// 128 x 128 logits: 128 query rows x the 128 keys of a tile in pass 1, the 128 keys of a tile x
+// a chunk of 128 query rows in pass 2.  Key tiles alternate between the two pairs of
+// warpgroups (each pair has its own issuing thread); within a pair the items of a tile
+// alternate between its two warpgroups, which start alternately from tile to tile.  A
+// warpgroup drains an item whole, four 32-column loads with the arithmetic in between, and
+// hands the buffer back after the last load, so the four warps that share an SM
+// sub-partition run out of step with one another.
 // The exponential is the scarce resource (16 MUFU results per clock per SM against 32 logits per
 // clock from the tensor cores), so a fixed share of the elements is evaluated on the FMA pipes
 // instead (range reduction + cubic polynomial, relative error 7.5e-5), and the surrounding
 // arithmetic uses the packed two-lane fp32 instructions to halve its issue slots.  Warpgroups
 // never synchronise inside a unit: pass 1 writes their statistics as separate partials; in
-// pass 2 a key tile belongs to one pair, whose two warpgroups add their per-key sums into the
-// zero-filled output with one reduction each (two addends, so the result does not depend on
-// their order).  More query rows than fit in shared memory are scored in several launches over
-// groups of rows (ScoreParams::row0), each adding into the same output.
+// pass 2 a key tile belongs to one pair, whose two warpgroups add their per-key sums (over the
+// chunks each of them drained) into the zero-filled output with one reduction each (two
+// addends, so the result does not depend on their order).  More query rows than fit in shared
+// memory are scored in several launches over groups of rows (ScoreParams::row0), each adding
+// into the same output.
 // The global key-tile space (layer, KV head, sequence, tile) is cut into equal contiguous
 // ranges, one per CTA.
 //
@@ -387,10 +390,10 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
   if (tid == 32) {
     // pass 1: one MMA thread, every buffer drained by all 16 epilogue warps;
     // pass 2: two MMA threads release a stage, a buffer is drained by the 8 warps of one pair
-    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], PASS == 1 ? 1 : 2); }
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 2); }
     mbar_init(q_full, 1);
-    mbar_init(q_empty, PASS == 1 ? 1 : 2);
-    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], PASS == 1 ? 16 : 8); }
+    mbar_init(q_empty, 2);
+    for (int i = 0; i < 4; ++i) { mbar_init(&t_full[i], 1); mbar_init(&t_empty[i], 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -403,8 +406,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
   const uint32_t tmem_base = *tmem_slot;
   const int n_kh = p.d / 64;                               // 64-element halves of the contraction
   const uint32_t q_half_bytes = (uint32_t)p.M_pad * 128u;
-  // K ring: [64-element half of the contraction][stage][128 keys x 128 bytes], so that two
-  // consecutive stages form one 256-key operand
+  // K ring: [64-element half of the contraction][stage][128 keys x 128 bytes]
   const uint32_t k_half_bytes = (uint32_t)p.n_stages * (128u * 128u);
 
   if (warp == 0) {
@@ -434,14 +436,6 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           for (int kh = 0; kh < n_kh; ++kh)
             tma_load_4d(dst + kh * k_half_bytes, &tm_k, kh * 64, row, sg.h, sg.l, &k_full[stage]);
         }
-        if (PASS == 1 && ok && (sg.nt & 1)) {
-          // pass 1 consumes stages in pairs: an odd segment is padded with an empty slot
-          const int stage = kit % p.n_stages;
-          ok = mbar_wait(&k_empty[stage], ((kit / p.n_stages) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive(&k_full[stage]);
-          ++kit;
-        }
       }
     }
   } else if (warp == 1 || warp == kMmaWarpB) {
@@ -449,14 +443,14 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     // Two issuing threads, one per warpgroup pair.  An issuing thread is a serial chain of
     // barrier waits and tcgen05.mma instructions (each holds the thread for about 60 cycles),
     // so one thread alone leaves the tensor pipe idle for more than half of the time.  Thread s
-    // feeds pair s only and owns that pair's two TMEM buffers (s and s + 2).  Both threads
+    // feeds pair s only: the buffers 2s and 2s + 1 of that pair's two warpgroups.  Both threads
     // wait for every key tile and commit to its "empty" barrier, whether or not they used it,
     // so that every phase of those barriers sees exactly two arrivals.
     if (lane == 0) {
       const int strm = warp == 1 ? 0 : 1;
       SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
       Seg sg;
-      uint32_t kit = 0, nseg = 0, j = 0;                    // j: items issued (pass 2: to my pair)
+      uint32_t kit = 0, nseg = 0;
       bool ok = true;
       const uint32_t idesc_full = make_idesc(128);
       const uint32_t idesc_last = make_idesc(PASS == 1 ? 128 : p.cw_last);
@@ -464,74 +458,46 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
       const uint32_t q_lo0 = desc_lo(smem_u32(q_sm)), k_lo0 = desc_lo(smem_u32(k_sm));
       const uint32_t q_half16 = q_half_bytes >> 4;
       const uint32_t k_half16 = k_half_bytes >> 4;
-      while (ok && (PASS == 2 || strm == 0) && seg_next(it, p, tp, sg)) {
+      uint32_t uses[2] = {0u, 0u};                            // items issued into each of my pair's two buffers
+      while (ok && seg_next(it, p, tp, sg)) {
         ok = mbar_wait(q_full, nseg & 1, abort_flag);
         if (!ok) break;
         ++nseg;
         tc_fence_after();
-        if (PASS == 1) {
-          // Work item = (two key tiles, block of 128 query rows): D[128 x 256] in one of two
-          // 256-column buffers, drained by all epilogue warps.  Half as many instructions per
-          // logit as with 128-key items, so one issuing thread keeps ahead of the epilogue.
-          for (int t = 0; t < sg.nt && ok; t += 2, kit += 2) {
-            const int stage = kit % p.n_stages;              // even: n_stages is even and segments use whole pairs
-            const uint32_t par = (kit / p.n_stages) & 1;
-            ok = mbar_wait(&k_full[stage], par, abort_flag) && mbar_wait(&k_full[stage + 1], par, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_lo = k_lo0 + stage * ((128 * 128) >> 4);
-            const uint32_t idesc = t + 1 < sg.nt ? make_idesc(256) : idesc_full;   // the padding slot holds no keys
-            for (int sub = 0; sub < n_sub; ++sub, ++j) {
-              const int buf = (int)(j & 1u);
-              ok = mbar_wait(&t_empty[buf], ((j >> 1) & 1) ^ 1, abort_flag);
+        // A key tile belongs to the pair with the parity of its index in the segment; within the
+        // pair, sub-item `sub` (a block of 128 query rows) of the pair's k-th tile goes to the
+        // warpgroup (sub + k) & 1, whose private 128-column buffer receives it.
+        for (int t = 0; t < sg.nt && ok; ++t, ++kit) {
+          const int stage = kit % p.n_stages;
+          ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_lo = k_lo0 + stage * ((128 * 128) >> 4);
+          if ((t & 1) == strm) {
+            for (int sub = 0; sub < n_sub; ++sub) {
+              const int h = (sub + (t >> 1)) & 1;
+              const int buf = strm * 2 + h;
+              ok = mbar_wait(&t_empty[buf], (uses[h] & 1) ^ 1, abort_flag);
               if (!ok) break;
+              ++uses[h];
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + buf * 256;
-              const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);      // 128 query rows of 128 bytes
+              const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
+              const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);
+              const uint32_t idesc = (PASS == 2 && sub == n_sub - 1) ? idesc_last : idesc_full;
 #pragma unroll
               for (int kh = 0; kh < 2; ++kh) {
                 if (kh < n_kh) {
 #pragma unroll
-                  for (int ks = 0; ks < 4; ++ks)
-                    tc_mma(d_tmem, desc_at(q_lo + kh * q_half16 + ks * 2), desc_at(k_lo + kh * k_half16 + ks * 2), idesc, (kh | ks) != 0);
+                  for (int ks = 0; ks < 4; ++ks) {
+                    if (PASS == 1) tc_mma(d_tmem, desc_at(q_lo + kh * q_half16 + ks * 2), desc_at(k_lo + kh * k_half16 + ks * 2), idesc, (kh | ks) != 0);
+                    else tc_mma(d_tmem, desc_at(k_lo + kh * k_half16 + ks * 2), desc_at(q_lo + kh * q_half16 + ks * 2), idesc, (kh | ks) != 0);
+                  }
                 }
               }
               tc_commit(&t_full[buf]);
             }
-            if (ok) { tc_commit(&k_empty[stage]); tc_commit(&k_empty[stage + 1]); }
           }
-        } else {
-          // The whole tile, all chunks of query rows, belongs to the pair with the parity of the
-          // tile's index in the segment, so that a key is reduced by one pair only.
-          for (int t = 0; t < sg.nt && ok; ++t, ++kit) {
-            const int stage = kit % p.n_stages;
-            ok = mbar_wait(&k_full[stage], (kit / p.n_stages) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_lo = k_lo0 + stage * ((128 * 128) >> 4);
-            if ((t & 1) == strm) {
-              for (int sub = 0; sub < n_sub; ++sub) {
-                const int buf = strm + 2 * (int)(j & 1u);
-                ok = mbar_wait(&t_empty[buf], ((j >> 1) & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                ++j;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BUFCOLS;
-                const uint32_t q_lo = q_lo0 + sub * ((128 * 128) >> 4);
-                const uint32_t idesc = (sub == n_sub - 1) ? idesc_last : idesc_full;
-#pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                  if (kh < n_kh) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                      tc_mma(d_tmem, desc_at(k_lo + kh * k_half16 + ks * 2), desc_at(q_lo + kh * q_half16 + ks * 2), idesc, (kh | ks) != 0);
-                  }
-                }
-                tc_commit(&t_full[buf]);
-              }
-            }
-            if (ok) tc_commit(&k_empty[stage]);      // arrives once my MMAs on this stage (if any) retire
-          }
+          if (ok) tc_commit(&k_empty[stage]);      // arrives once my MMAs on this stage (if any) retire
         }
         if (ok) tc_commit(q_empty);
       }
@@ -539,7 +505,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
   } else if (warp < kMmaWarpB) {
     // ------------------------------------------------ epilogue --------
     const int wg = (warp - 2) >> 2;                        // warpgroup 0..3
-    const int pair = wg >> 1;                              // pairs take alternate work items
+    const int pair = wg >> 1;                              // pairs take alternate key tiles
     const int half = wg & 1;                               // column half of the pair's buffer
     const int quarter = warp & 3;                          // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
@@ -547,53 +513,54 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
     SegIter it = seg_begin(p, tp, gridDim.x, blockIdx.x);
     Seg sg;
-    uint32_t bit = 0;
     bool ok = true;
     uint32_t ra[32];
+    uint32_t used = 0;                                       // items drained from my warpgroup's buffer
+    const uint32_t my_taddr = lane_base + wg * BUFCOLS;
     if (PASS == 1) {
-      // Work item = 128 query rows (on lanes) x 256 keys (two tiles) in one of two 256-column
-      // buffers; every warpgroup owns 64 of its key columns.
+      // Work item = 128 query rows (on lanes) x the 128 keys of a tile, all of it mine.
       const int n_mt = p.M_pad / 128;
       float mrun[kMaxMTiles], zrun[kMaxMTiles];
       while (ok && seg_next(it, p, tp, sg)) {
 #pragma unroll
         for (int i = 0; i < kMaxMTiles; ++i) { mrun[i] = -INFINITY; zrun[i] = 0.f; }
-        for (int t = 0; t < sg.nt && ok; t += 2) {
-          const int n_item = t + 1 < sg.nt ? 2 * kTileKeys : kTileKeys;            // the last item of an odd segment is one tile
-          const int key0 = (sg.t0 + t) * kTileKeys;                                // first key of the item
-          const int nvh = min(n_item, sg.n - key0) - wg * 64;                      // valid keys in my 64 columns
-          const bool in_window = p.causal && key0 + n_item > sg.n - p.n_window;    // warp-uniform
-          const bool plain = nvh >= 64 && !in_window;
-          for (int mt = 0; mt < n_mt; ++mt, ++bit) {
-            const int buf = (int)(bit & 1u);
-            ok = mbar_wait(&t_full[buf], (bit >> 1) & 1, abort_flag);
+        for (int t = pair; t < sg.nt && ok; t += 2) {
+          const int key0 = (sg.t0 + t) * kTileKeys;                                // first key of the tile
+          const int nv = min(kTileKeys, sg.n - key0);                              // valid keys of the tile
+          const bool in_window = p.causal && key0 + kTileKeys > sg.n - p.n_window;    // warp-uniform
+          const bool plain = nv >= kTileKeys && !in_window;
+          for (int mt = ((t >> 1) + half) & 1; mt < n_mt && ok; mt += 2) {
+            ok = mbar_wait(&t_full[wg], used & 1, abort_flag);
             if (!ok) break;
+            ++used;
             tc_fence_after();
             float m = mrun[mt], z = zrun[mt];
-            const uint32_t taddr = lane_base + buf * 256 + wg * 64;
             if (plain) {
-              // all 64 of my columns are keys every row sees: no masks, no per-row arithmetic
-              tmem_ld32(taddr, ra);
+              // every row sees all 128 keys: no masks, no per-row arithmetic
+              tmem_ld32(my_taddr, ra);
               stats_update<false>(ra, 32, p.a, m, z);
-              tmem_ld32(taddr + 32, ra);
+              tmem_ld32(my_taddr + 32, ra);
+              stats_update<false>(ra, 32, p.a, m, z);
+              tmem_ld32(my_taddr + 64, ra);
+              stats_update<false>(ra, 32, p.a, m, z);
+              tmem_ld32(my_taddr + 96, ra);
               tc_fence_before();
-              arrive_lane0(&t_empty[buf], lane);               // all reads done: the buffer can be refilled
+              arrive_lane0(&t_empty[wg], lane);               // all reads done: the buffer can be refilled
               stats_update<false>(ra, 32, p.a, m, z);
             } else {
-              int vis = nvh, vis2 = 0;                         // keys of my 64 columns that this thread's row may see
-              if (nvh > 0) {
-                if (in_window) {
-                  const int rr = (p.row0 + mt * 128 + row_in_tile) % p.R;
-                  if (rr < p.n_window) vis = min(nvh, max(sg.n - p.n_window + rr, 0) + 1 - (key0 + wg * 64));
-                }
-                tmem_ld32(taddr, ra);
-                if (vis > 0) stats_update<true>(ra, min(vis, 32), p.a, m, z);
-                if (nvh > 32) tmem_ld32(taddr + 32, ra);
-                vis2 = vis - 32;
+              int vis = nv;                                    // keys of the tile that this thread's row may see
+              if (in_window) {
+                const int rr = (p.row0 + mt * 128 + row_in_tile) % p.R;
+                if (rr < p.n_window) vis = min(nv, max(sg.n - p.n_window + rr, 0) + 1 - key0);
+              }
+#pragma unroll 1
+              for (int c = 0; c < 4; ++c) {
+                if (c * 32 >= nv) break;                                    // warp-uniform
+                tmem_ld32(my_taddr + c * 32, ra);
+                if (vis - c * 32 > 0) stats_update<true>(ra, min(vis - c * 32, 32), p.a, m, z);
               }
               tc_fence_before();
-              arrive_lane0(&t_empty[buf], lane);
-              if (nvh > 32 && vis2 > 0) stats_update<true>(ra, min(vis2, 32), p.a, m, z);
+              arrive_lane0(&t_empty[wg], lane);
             }
             mrun[mt] = m;
             zrun[mt] = z;
@@ -611,10 +578,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
       }
     } else {
-      // Work item = one key tile (keys on lanes) with all its chunks of 128 query rows; this
-      // warpgroup owns half of every chunk's columns.
+      // Work item = one key tile (keys on lanes) x one chunk of 128 query rows, all of it mine; the
+      // chunks of a tile alternate between the two warpgroups of the pair.
       const float2 a2 = splat2(p.a);
-      uint32_t j = 0;                                        // this pair's item counter
       // Every epilogue thread passes the two barriers of every segment, also after a wait has
       // given up, so that no warp is left waiting at them.
       while (seg_next(it, p, tp, sg)) {
@@ -627,28 +593,30 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           float2 acc[2] = {splat2(0.f), splat2(0.f)};
           const int key = (sg.t0 + t) * kTileKeys + row_in_tile;
           const bool in_window = p.causal && (sg.t0 + t + 1) * kTileKeys > sg.n - p.n_window;   // warp-uniform
-          for (int ch = 0; ch < p.n_chunks; ++ch, ++j) {
-            const int buf = pair + 2 * (int)(j & 1u);
-            ok = mbar_wait(&t_full[buf], (j >> 1) & 1, abort_flag);
+          bool any = false;
+          for (int ch = ((t >> 1) + half) & 1; ch < p.n_chunks; ch += 2) {
+            ok = mbar_wait(&t_full[wg], used & 1, abort_flag);
             if (!ok) break;
+            ++used;
+            any = true;
             tc_fence_after();
-            const int hw = (ch == p.n_chunks - 1 ? p.cw_last : 128) >> 1;     // my columns: 32 or 64
-            const uint32_t taddr = lane_base + buf * BUFCOLS + half * hw;
-            const float* negc = c_sm + ch * 128 + half * hw;
-            const int row0 = p.row0 + ch * 128 + half * hw;     // query row of my first column
-            tmem_ld32(taddr, ra);
-            if (hw > 32) {
-              if (!in_window) prob_accumulate<MAXRED>(ra, negc, a2, acc);
-              else prob_accumulate_causal<MAXRED>(ra, negc, p.a, acc, row0, p.R, p.n_window, sg.n, key);
-              tmem_ld32(taddr + 32, ra);
+            const int cw = ch == p.n_chunks - 1 ? p.cw_last : 128;            // my columns: 64 or 128
+            const float* negc = c_sm + ch * 128;
+            const int row0 = p.row0 + ch * 128;                 // query row of my first column
+            const int nb = cw >> 5;                             // blocks of 32 columns: 2 or 4
+#pragma unroll 1
+            for (int c = 0; c < nb; ++c) {
+              tmem_ld32(my_taddr + c * 32, ra);
+              if (c == nb - 1) {
+                tc_fence_before();
+                arrive_lane0(&t_empty[wg], lane);
+              }
+              if (!in_window) prob_accumulate<MAXRED>(ra, negc + c * 32, a2, acc);
+              else prob_accumulate_causal<MAXRED>(ra, negc + c * 32, p.a, acc, row0 + c * 32, p.R, p.n_window, sg.n, key);
             }
-            tc_fence_before();
-            arrive_lane0(&t_empty[buf], lane);
-            if (!in_window) prob_accumulate<MAXRED>(ra, hw > 32 ? negc + 32 : negc, a2, acc);
-            else prob_accumulate_causal<MAXRED>(ra, hw > 32 ? negc + 32 : negc, p.a, acc, hw > 32 ? row0 + 32 : row0, p.R, p.n_window, sg.n, key);
           }
           if (!ok) break;
-          if (key < sg.n) {
+          if (any && key < sg.n) {
             // The output was zero-filled; the two warpgroups of the pair contribute once per key.
             const float v0 = acc[0].x, v1 = acc[0].y, v2 = acc[1].x, v3 = acc[1].y;
             if (MAXRED) {
@@ -849,7 +817,6 @@ SPEC_EXPORT int32_t spec_score(const spec_problem* pr, const void* q, const void
     const int smem_max = 227 * 1024;
     int stages = (smem_max - (int)p.q_bytes - small) / (int)p.stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
-    stages &= ~1;                                          // pass 1 consumes the ring two stages at a time
     if (stages < 2) return fail(SPEC_ERR_UNSUPPORTED, "not enough shared memory for two key stages (%d rows, head_dim=%d)", p.M, d);
     p.n_stages = stages;
     int smem = stages * (int)p.stage_bytes + (int)p.q_bytes + small;
