@@ -64,11 +64,18 @@ struct UnitGeom {
   int cand_cap;
 };
 
+__device__ __forceinline__ UnitGeom unit_geom_of(const StreamParams& p, int s, int row);
+
 __device__ __forceinline__ UnitGeom unit_geom(const StreamParams& p, int unit) {
+  const int rows = p.H * p.L;
+  return unit_geom_of(p, unit / rows, unit % rows);
+}
+
+// row = layer * H + head
+__device__ __forceinline__ UnitGeom unit_geom_of(const StreamParams& p, int s, int row) {
   UnitGeom g;
-  g.h = unit % p.H;
-  g.l = (unit / p.H) % p.L;
-  g.s = unit / (p.H * p.L);
+  g.s = s;
+  g.l = g.h = 0;                                          // only their combination, `row`, is used
   seq_range(p.cu, p.n_in, g.s, g.begin, g.n);
   g.over = g.n > p.max_len;
   if (g.over) g.n = 0;
@@ -76,9 +83,9 @@ __device__ __forceinline__ UnitGeom unit_geom(const StreamParams& p, int unit) {
   g.e = g.n - g.forced;
   g.take[0] = max(min(p.c_max - g.forced, g.e), 0);
   g.take[1] = max(min(p.n_vert, g.e), 0);
-  g.src = p.scores + ((int64_t)g.l * p.H + g.h) * p.T + g.begin;
+  g.src = p.scores + (int64_t)row * p.T + g.begin;
   // even, so that a segment starts on a 16-byte boundary
-  g.cand_off = ((int64_t)g.l * p.H + g.h) * p.row_entries + ((g.begin + 1) & ~1) + (int64_t)g.s * kSelCandSlack;
+  g.cand_off = (int64_t)row * p.row_entries + ((g.begin + 1) & ~1) + (int64_t)g.s * kSelCandSlack;
   g.cand_cap = g.n + kSelCandSlack;
   return g;
 }
@@ -172,12 +179,11 @@ struct SweepItem {
   bool active, bulk;
 };
 
-__device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int64_t item) {
+__device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int s, int row, int chunk_id) {
   SweepItem t;
-  const int unit = (int)(item / p.chunks_max);
-  t.chunk_id = (int)(item % p.chunks_max);
-  t.g = unit_geom(p, unit);
-  t.hd = p.head + (int64_t)unit * p.head_words;
+  t.chunk_id = chunk_id;
+  t.g = unit_geom_of(p, s, row);
+  t.hd = p.head + ((int64_t)s * (p.H * p.L) + row) * p.head_words;
   t.floor_key = 0;                                         // read by the caller once the copy is under way
   t.mis = (int)((reinterpret_cast<uintptr_t>(t.g.src) >> 2) & 3u);
   t.X = t.g.e + t.mis;                                     // x = position + mis: multiples of four are 16-byte boundaries
@@ -195,15 +201,44 @@ __device__ __forceinline__ SweepItem sweep_item(const StreamParams& p, int64_t i
   return t;
 }
 
-// One CTA per item.  Eight small CTAs share an SM, so that the bulk copies of some overlap the
-// pooling of others (a persistent, double-buffered variant with fewer resident warps was slower).
+// Pools my warp's steps straight from shared memory; bit 4k + u of the returned mask marks the
+// candidates (pooled value at or above the floor) among my four positions of step k.  EDGE: the
+// chunk holds slots that are not positions of the unit (only the chunks at either end do).
+template <bool EDGE>
+__device__ __forceinline__ uint32_t sweep_steps(const SweepItem& t, const float* raw, float floor_f, int warp, int lane) {
+  const float4* base4 = reinterpret_cast<const float4*>(raw + 4);
+  uint32_t mask = 0;
+#pragma unroll
+  for (int k = 0; k < kMaxStepsPerWarp; ++k) {
+    const int st = warp + k * kSweepWarps;
+    if (st < t.n_steps) {
+      const float4* at = base4 + st * 32 + lane;
+      const float4 pv = at[-1], cv = at[0], nv = at[1];
+      const float x[10] = {pv.y, pv.z, pv.w, cv.x, cv.y, cv.z, cv.w, nv.x, nv.y, nv.z};
+      float t3[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t3[i] = fmax3(x[i], x[i + 1], x[i + 2]);
+      const int pp0 = t.x0 + st * 128 + lane * 4 - t.mis;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        bool c = !(fmax3(t3[u], t3[u + 3], x[u + 6]) < floor_f);
+        if (EDGE) c = c && pp0 + u >= 0 && pp0 + u < t.g.e;
+        if (c) mask |= 1u << (4 * k + u);
+      }
+    }
+  }
+  return mask;
+}
+
+// One CTA per (unit, chunk).  Many small CTAs share an SM, so that the bulk copies of some overlap
+// the pooling of others (fatter CTAs, and persistent double-buffered ones, were slower).
 __global__ void __launch_bounds__(kSweepThreads, 16) stream_sweep_kernel(const StreamParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __shared__ int wsum[kSweepWarps];
   __shared__ uint64_t mbar;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  SweepItem t = sweep_item(p, blockIdx.x);
+  SweepItem t = sweep_item(p, blockIdx.z, blockIdx.y, blockIdx.x);
   if (!t.active) return;
   float* raw = reinterpret_cast<float*>(smem_raw);
   const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&mbar);
@@ -239,39 +274,11 @@ __global__ void __launch_bounds__(kSweepThreads, 16) stream_sweep_kernel(const S
     }
   }
   if (t.floor_key == kNoSelection) return;
-  // ---- pooled maxima straight from shared memory, kept in registers; warp w owns steps w, w + 2, ...
-  // Only the chunks at either end of the unit hold slots that are not positions.
   const float floor_f = key_to_float(t.floor_key);
-  const float4* base4 = reinterpret_cast<const float4*>(raw + 4);
   const bool edge = t.x0 < t.mis || t.x0 + t.n_steps * 128 > t.X;
-  float pooled[kMaxStepsPerWarp][4];
-  int mine = 0;
-#pragma unroll
-  for (int k = 0; k < kMaxStepsPerWarp; ++k) {
-    const int st = warp + k * kSweepWarps;
-    if (st < t.n_steps) {
-      const float4* at = base4 + st * 32 + lane;
-      const float4 pv = at[-1], cv = at[0], nv = at[1];
-      const float x[10] = {pv.y, pv.z, pv.w, cv.x, cv.y, cv.z, cv.w, nv.x, nv.y, nv.z};
-      float t3[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) t3[i] = fmax3(x[i], x[i + 1], x[i + 2]);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) pooled[k][u] = fmax3(t3[u], t3[u + 3], x[u + 6]);
-      if (edge) {
-        const int pp0 = t.x0 + st * 128 + lane * 4 - t.mis;
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (pp0 + u < 0 || pp0 + u >= t.g.e) pooled[k][u] = __uint_as_float(0xFFFFFFFFu);   // not a position: never a candidate
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) mine += !(pooled[k][u] < floor_f) && __float_as_uint(pooled[k][u]) != 0xFFFFFFFFu;
-    } else {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) pooled[k][u] = __uint_as_float(0xFFFFFFFFu);
-    }
-  }
+  uint32_t mask = edge ? sweep_steps<true>(t, raw, floor_f, warp, lane) : sweep_steps<false>(t, raw, floor_f, warp, lane);
   // ---- my candidates go to my own segment of the unit's array, their number to the unit's header
+  const int mine = __popc(mask);
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -288,16 +295,15 @@ __global__ void __launch_bounds__(kSweepThreads, 16) stream_sweep_kernel(const S
     n_cta += c;
   }
   if (tid == 0) t.hd[4 + t.chunk_id] = n_cta;              // a segment is as long as the chunk: it cannot overflow
-  if (mine == 0) return;
+  // Few positions are candidates: each lane walks its own, pooling them again from the staged scores.
   uint2* dst = p.cand + t.g.cand_off + (int64_t)t.chunk_id * p.chunk + before;
-#pragma unroll
-  for (int k = 0; k < kMaxStepsPerWarp; ++k) {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float v = pooled[k][u];
-      if (!(v < floor_f) && __float_as_uint(v) != 0xFFFFFFFFu)
-        *dst++ = make_uint2(to_key(v), (uint32_t)(t.x0 + (warp + k * kSweepWarps) * 128 + lane * 4 + u - t.mis));
-    }
+  while (mask) {
+    const int b = __ffs(mask) - 1;
+    mask &= mask - 1;
+    const int j = (warp + (b >> 2) * kSweepWarps) * 128 + lane * 4 + (b & 3);     // position within the chunk
+    const float* w7 = raw + 4 + j - 3;
+    const float v = fmax3(fmax3(w7[0], w7[1], w7[2]), fmax3(w7[3], w7[4], w7[5]), w7[6]);
+    *dst++ = make_uint2(to_key(v), (uint32_t)(t.x0 + j - t.mis));
   }
 }
 
@@ -395,19 +401,66 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         // ---- exact threshold among the candidates
         uint32_t prefix = 0, mask = 0;
         int remaining = tk;
-        for (int pass = 0; pass < 3; ++pass) {
+        int first_pass = 0;
+        {
+          // The leading 11 bits first, without a histogram: every candidate is at or above the floor,
+          // so they fall into a few bins from the floor's bin up.  Every thread counts the eight
+          // lowest of those bins (and everything higher together) in registers; the sums over the
+          // CTA locate the digit unless the threshold lies higher still (then the histogram pass).
+          const uint32_t fb = (uint32_t)hd[0] >> 21;
+          int c8[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+          for (int i = tid; i < n_cand; i += kSelThreads) {
+            const uint2 ck = cand[i];
+            if (ck.y == kNoSelection) continue;
+            const uint32_t d = (ck.x >> 21) - fb;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) c8[b] += d == (uint32_t)b;
+            c8[8] += d >= 8u;
+          }
+#pragma unroll
+          for (int b = 0; b < 9; ++b) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) c8[b] += __shfl_xor_sync(0xffffffffu, c8[b], o);
+          }
+          int* wc = reinterpret_cast<int*>(hist);             // [kSelWarps][9]
+          __syncthreads();
+          if ((tid & 31) == 0) {
+#pragma unroll
+            for (int b = 0; b < 9; ++b) wc[(tid >> 5) * 9 + b] = c8[b];
+          }
+          __syncthreads();
+          int tot[9];
+#pragma unroll
+          for (int b = 0; b < 9; ++b) {
+            tot[b] = 0;
+            for (int w = 0; w < kSelWarps; ++w) tot[b] += wc[w * 9 + b];
+          }
+          __syncthreads();
+          if (tot[8] < remaining) {
+            int above = tot[8], b = 7;
+            for (; b > 0; --b) {
+              if (above + tot[b] >= remaining) break;
+              above += tot[b];
+            }
+            remaining -= above;
+            prefix = (fb + (uint32_t)b) << 21;
+            mask = 2047u << 21;
+            first_pass = 1;
+          }
+        }
+        for (int pass = first_pass; pass < 3; ++pass) {
           const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
           const uint32_t dmask = pass == 2 ? 1023u : 2047u;
           for (int i = tid; i < kStreamBins; i += kSelThreads) hist[i] = 0;
           __syncthreads();
           for (int i0 = 0; i0 < n_cand; i0 += kSelThreads) {
-            // lanes of a warp with the same digit add once: the candidates share their leading bits
             const int i = i0 + tid;
             const uint2 ck = i < n_cand ? cand[i] : make_uint2(0u, kNoSelection);
             const uint32_t kk = ck.x;
             const bool in = ck.y != kNoSelection && (kk & mask) == prefix;
             const uint32_t dgt = (kk >> shift) & dmask;
             if (pass == 0) {
+              // lanes of a warp with the same digit add once: the candidates share their leading bits
               const uint32_t act = __ballot_sync(0xffffffffu, in);
               if (in) {
                 const uint32_t same = __match_any_sync(act, dgt);
@@ -507,7 +560,6 @@ int run_stream_topk(const spec_problem* pr, const float* scores, int c_max, int 
     p.held_cap = (int)(room & ~(int64_t)3);
   }
   const size_t smem_finish = stream_finish_bytes(p.bitmap_words, p.held_cap);
-  if (n_units * p.chunks_max > 0x7fffffffLL) return SPEC_OK;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   p.head = reinterpret_cast<int32_t*>(ws + wp.sel_head_off);
   p.head_words = wp.sel_head_words;
@@ -526,7 +578,9 @@ int run_stream_topk(const spec_problem* pr, const float* scores, int c_max, int 
   }
   sample_floor_kernel<<<(unsigned)n_units, kSelThreads, 0, st>>>(p);
   SPEC_CUDA_OK(cudaGetLastError());
-  stream_sweep_kernel<<<(unsigned)(n_units * p.chunks_max), kSweepThreads, smem_sweep, st>>>(p);
+  if (pr->n_layers * pr->n_kv_heads > 65535) return SPEC_OK;   // rows are a grid dimension of the sweep
+  const dim3 sweep_grid((unsigned)p.chunks_max, (unsigned)(pr->n_layers * pr->n_kv_heads), (unsigned)pr->n_seq);
+  stream_sweep_kernel<<<sweep_grid, kSweepThreads, smem_sweep, st>>>(p);
   SPEC_CUDA_OK(cudaGetLastError());
   stream_finish_kernel<<<(unsigned)n_units, kSelThreads, smem_finish, st>>>(p);
   SPEC_CUDA_OK(cudaGetLastError());
