@@ -102,6 +102,9 @@ __global__ void __launch_bounds__(kSelThreads) sample_floor_kernel(const StreamP
   __shared__ int wsum[32];
   __shared__ int out2[4];
   const int unit = blockIdx.x, tid = threadIdx.x;
+  // The sweep is launched as a programmatic dependent: its CTAs may start now and issue the copies of
+  // their chunks; they wait for this grid to finish before they read the floor.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const UnitGeom g = unit_geom(p, unit);
   const int tk = max(g.take[0], g.take[1]);
   const bool selects = (g.take[0] > 0 && g.take[0] < g.e) || (g.take[1] > 0 && g.take[1] < g.e);
@@ -261,7 +264,8 @@ __global__ void __launch_bounds__(kSweepThreads, 16) stream_sweep_kernel(const S
   }
   // The floor is fetched while the copy is in flight.  A unit that keeps everything or nothing needs no sweep,
   // but its copy is awaited all the same: shared memory must not be given up with a copy under way.
-  t.floor_key = (uint32_t)__ldg(t.hd);
+  asm volatile("griddepcontrol.wait;" ::: "memory");     // the floors are written by the grid before this one
+  t.floor_key = (uint32_t)__ldcg(t.hd);
   __syncthreads();                                         // the barrier is initialised; the edges are in place
   if (t.bulk) {
     uint32_t ok = 0;
@@ -325,6 +329,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
   const int unit = blockIdx.x;
   const UnitGeom g = unit_geom(p, unit);
   const int32_t* hd = p.head + (int64_t)unit * p.head_words;
+  asm volatile("griddepcontrol.wait;" ::: "memory");     // the candidates are written by the grid before this one
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);
   uint2* held = reinterpret_cast<uint2*>(hist + kStreamBins);
   uint32_t* map_gt = reinterpret_cast<uint32_t*>(held + p.held_cap);
@@ -408,15 +413,17 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
           // lowest of those bins (and everything higher together) in registers; the sums over the
           // CTA locate the digit unless the threshold lies higher still (then the histogram pass).
           const uint32_t fb = (uint32_t)hd[0] >> 21;
-          int c8[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+          // nine 7-bit counters packed in one word pair per thread (a thread sees at most
+          // held_cap / 512 < 128 candidates)
+          unsigned long long packed = 0;
           for (int i = tid; i < n_cand; i += kSelThreads) {
             const uint2 ck = cand[i];
             if (ck.y == kNoSelection) continue;
-            const uint32_t d = (ck.x >> 21) - fb;
-#pragma unroll
-            for (int b = 0; b < 8; ++b) c8[b] += d == (uint32_t)b;
-            c8[8] += d >= 8u;
+            packed += 1ull << (7u * min((ck.x >> 21) - fb, 8u));
           }
+          int c8[9];
+#pragma unroll
+          for (int b = 0; b < 9; ++b) c8[b] = (int)((packed >> (7 * b)) & 127ull);
 #pragma unroll
           for (int b = 0; b < 9; ++b) {
 #pragma unroll
@@ -480,7 +487,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         const int need_eq = remaining;
         // ---- winners and ties into position bitmaps, then out in ascending position
         const int n_words = (g.e + 31) >> 5;
-        for (int w = tid; w < n_words; w += kSelThreads) { map_gt[w] = 0; map_eq[w] = 0; }
+        {
+          uint4* z4 = reinterpret_cast<uint4*>(map_gt);      // both bitmaps, adjacent, whole 16-byte words
+          const int n4 = (p.bitmap_words + ((n_words + 3) & ~3)) >> 2;
+          for (int w = tid; w < n4; w += kSelThreads) z4[w] = make_uint4(0u, 0u, 0u, 0u);
+        }
         __syncthreads();
         for (int i = tid; i < n_cand; i += kSelThreads) {
           const uint2 c = cand[i];
@@ -491,7 +502,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         __syncthreads();
         // Output rank of a position = winners (and ties) before it: an exclusive count per group of
         // a few words, kept where the histogram was, plus the words of its own group up to its bit.
-        const int gw = (n_words + 2 * kSelThreads - 1) / (2 * kSelThreads);   // words per group, two groups per thread
+        int gshift = 0;                                                          // words per group = 2^gshift, two groups per thread
+        while ((2 * kSelThreads << gshift) < n_words) ++gshift;
+        const int gw = 1 << gshift;
         int* grp_gt = reinterpret_cast<int*>(hist);
         int* grp_eq = grp_gt + 2 * kSelThreads;
         int gt0 = 0, eq0 = 0, gt1 = 0, eq1 = 0;
@@ -508,10 +521,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         for (int i = tid; i < n_cand; i += kSelThreads) {
           const uint2 c = cand[i];
           if (c.x < T || c.y == kNoSelection) continue;
-          const int w = (int)(c.y >> 5), grp = w / gw;
+          const int w = (int)(c.y >> 5), grp = w >> gshift;
           const uint32_t below = (1u << (c.y & 31)) - 1u;
           int g_before = grp_gt[grp] + __popc(map_gt[w] & below), q_before = grp_eq[grp] + __popc(map_eq[w] & below);
-          for (int ww = grp * gw; ww < w; ++ww) { g_before += __popc(map_gt[ww]); q_before += __popc(map_eq[ww]); }
+          for (int ww = grp << gshift; ww < w; ++ww) { g_before += __popc(map_gt[ww]); q_before += __popc(map_eq[ww]); }
           if (c.x > T) idx[g_before + min(q_before, need_eq)] = (int32_t)c.y;
           else if (q_before < need_eq) idx[g_before + q_before] = (int32_t)c.y;
         }
@@ -580,10 +593,23 @@ int run_stream_topk(const spec_problem* pr, const float* scores, int c_max, int 
   SPEC_CUDA_OK(cudaGetLastError());
   if (pr->n_layers * pr->n_kv_heads > 65535) return SPEC_OK;   // rows are a grid dimension of the sweep
   const dim3 sweep_grid((unsigned)p.chunks_max, (unsigned)(pr->n_layers * pr->n_kv_heads), (unsigned)pr->n_seq);
-  stream_sweep_kernel<<<sweep_grid, kSweepThreads, smem_sweep, st>>>(p);
-  SPEC_CUDA_OK(cudaGetLastError());
-  stream_finish_kernel<<<(unsigned)n_units, kSelThreads, smem_finish, st>>>(p);
-  SPEC_CUDA_OK(cudaGetLastError());
+  // The sweep and the finishing kernel are programmatic dependents of the kernel before them: they are
+  // launched while it still runs and wait, in the kernel, where they first need its results.
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = st;
+  cfg.attrs = pdl;
+  cfg.numAttrs = 1;
+  cfg.gridDim = sweep_grid;
+  cfg.blockDim = dim3(kSweepThreads);
+  cfg.dynamicSmemBytes = smem_sweep;
+  SPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, stream_sweep_kernel, p));
+  cfg.gridDim = dim3((unsigned)n_units);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem_finish;
+  SPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, stream_finish_kernel, p));
   *done = true;
   return SPEC_OK;
 }
