@@ -42,6 +42,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # makes the figure stale and it is reported as null.
 NCU_TRAFFIC = {
     # workload index -> {kernel group: (bytes per layer, source files, hash of those sources)}
+    # profiles/score_kernel_c2.md (2 layers) and profiles/select_and_gather_c2.md (8 layers)
+    2: {"score": ((542.008064e6 + 7.79392e6 + 550.035456e6 + 11.079168e6) / 2, ["score.cu"], "d44fc0da3556a83b"),
+        "select": ((8.40576e6 + 33.587712e6 + 0.007168e6 + 3.372544e6) / 8, ["select_stream.cu", "select_common.cuh"], "1c90281812721d22"),
+        "gather": ((67.677696e6 + 13.709824e6) / 8, ["compact.cu"], "4de11f4bd31ee049")},
 }
 
 
@@ -473,11 +477,14 @@ def main(argv=None):
                 "algorithmic_bytes": work["score_hbm_bytes"], "traffic": ncu_traffic(args.config, "score", st.L)}
     hbm_bytes = work["select_bytes"] + work["gather_bytes"]
     gbs = hbm_bytes / ((t_select + t_gather) * 1e-3) / 1e9
-    roofline_hbm = {"bound": "hbm", "kernel": "pool_topk_kernel + compact_kernel" if not st.specpc else "token_reduce + specpc_keep",
+    roofline_hbm = {"bound": "hbm", "kernel": ("sample_floor + stream_sweep + stream_finish + compact_bulk" if not st.specpc
+                                                 else "token_reduce + cluster_select"),
                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": peak_src + " (copy)", "ms_select": t_select, "ms_gather": t_gather,
                     "gather_gbs": (work["gather_bytes"] / (t_gather * 1e-3) / 1e9) if t_gather > 0 and work["gather_bytes"] else None,
                     "algorithmic_bytes": hbm_bytes,
+                    "traffic_note": "DRAM bytes under ncu on a small case, scaled by layers; gathered rows still in L2 when the "
+                                    "capture ended are not in it",
                     "traffic": (None if st.specpc or ncu_traffic(args.config, "select", st.L) is None or ncu_traffic(args.config, "gather", st.L) is None
                                 else ncu_traffic(args.config, "select", st.L) + ncu_traffic(args.config, "gather", st.L))}
 
