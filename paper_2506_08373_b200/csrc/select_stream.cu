@@ -9,7 +9,7 @@
 //      That key is a floor under the final threshold with overwhelming probability, and it does
 //      not depend on where in the unit the large scores sit (rising, falling or concentrated
 //      scores cost the same).
-//   2. stream_sweep_kernel, one small CTA per (unit, chunk of 4096 positions), eight to an SM: the
+//   2. stream_sweep_kernel, one small CTA per (unit, chunk of 2048 positions), sixteen to an SM: the
 //      chunk is staged in shared memory with one bulk asynchronous copy and pooled from there
 //      (three 16-byte reads per four positions, nothing written back); the positions at or above
 //      the floor go, as (key, position) pairs, to the chunk's own segment of the unit's candidate
@@ -324,9 +324,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __shared__ int wsum[32];
   __shared__ int out2[4];
+  __shared__ int lead[2][9];                               // per budget: candidates per leading-digit bin above the floor's
   __shared__ uint64_t mbar;
   const int tid = threadIdx.x;
   const int unit = blockIdx.x;
+  if (tid < 18) (&lead[0][0])[tid] = 0;
   const UnitGeom g = unit_geom(p, unit);
   const int32_t* hd = p.head + (int64_t)unit * p.head_words;
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the candidates are written by the grid before this one
@@ -346,8 +348,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
     const int my_cnt = (raw_cnt + 1) & ~1;                 // rounded up to a whole 16 bytes
     int total;
     const int mine_at = block_exclusive_scan(my_cnt, wsum, total);
-    __syncthreads();
-    block_exclusive_scan(raw_cnt, wsum, n_real);
+    n_real = total - __syncthreads_count(raw_cnt & 1);     // every odd count was rounded up by one
     failed = failed || total > p.held_cap;
     if (!failed) {
       // One bulk asynchronous copy per chunk, all in flight together.  Bulk copies move multiples of
@@ -365,6 +366,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
                      ::"r"((uint32_t)__cvta_generic_to_shared(held + mine_at)), "l"(segs + (int64_t)tid * p.chunk),
                        "r"((uint32_t)my_cnt * 8u), "r"(bar_a) : "memory");
       }
+      // while the copies are in flight: both position bitmaps (adjacent, whole 16-byte words) are cleared
+      {
+        uint4* z4 = reinterpret_cast<uint4*>(map_gt);
+        const int n4 = (p.bitmap_words + ((((g.e + 31) >> 5) + 3) & ~3)) >> 2;
+        for (int w = tid; w < n4; w += kSelThreads) z4[w] = make_uint4(0u, 0u, 0u, 0u);
+      }
       uint32_t ok = total == 0;
       for (uint32_t tries = 0; tries < (1u << 20) && !ok; ++tries)
         asm volatile("{\n.reg .pred q;\nmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\nselp.u32 %0, 1, 0, q;\n}"
@@ -380,6 +387,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
   }
   const uint2* cand = held;
   const int n_budgets = p.n_vert > 0 ? 2 : 1;
+  bool maps_dirty = false;
   for (int b = 0; b < n_budgets; ++b) {
     int32_t* idx = b == 0 ? p.idx_out + (int64_t)unit * p.c_max : p.vert_out + (int64_t)unit * p.n_vert;
     int32_t* cnt = b == 0 ? p.count_out : p.vert_count_out;
@@ -392,6 +400,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         __syncthreads();
         // generic selection: pooled keys recomputed from global memory in every pass
         SelectScratch sc;
+        maps_dirty = true;
         sc.hist = map_gt;
         sc.misc = reinterpret_cast<int*>(sc.hist + kSelWarps * 256);
         KeySource key;
@@ -415,34 +424,23 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
           const uint32_t fb = (uint32_t)hd[0] >> 21;
           // nine 7-bit counters packed in one word pair per thread (a thread sees at most
           // held_cap / 512 < 128 candidates)
+          int* lead_b = lead[b];
           unsigned long long packed = 0;
           for (int i = tid; i < n_cand; i += kSelThreads) {
             const uint2 ck = cand[i];
             if (ck.y == kNoSelection) continue;
             packed += 1ull << (7u * min((ck.x >> 21) - fb, 8u));
           }
-          int c8[9];
-#pragma unroll
-          for (int b = 0; b < 9; ++b) c8[b] = (int)((packed >> (7 * b)) & 127ull);
+          // one warp-wide reduction per counter, one shared-memory addition per warp and counter
 #pragma unroll
           for (int b = 0; b < 9; ++b) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) c8[b] += __shfl_xor_sync(0xffffffffu, c8[b], o);
-          }
-          int* wc = reinterpret_cast<int*>(hist);             // [kSelWarps][9]
-          __syncthreads();
-          if ((tid & 31) == 0) {
-#pragma unroll
-            for (int b = 0; b < 9; ++b) wc[(tid >> 5) * 9 + b] = c8[b];
+            const uint32_t v = __reduce_add_sync(0xffffffffu, (uint32_t)((packed >> (7 * b)) & 127ull));
+            if ((tid & 31) == 0 && v) atomicAdd(&lead_b[b], (int)v);
           }
           __syncthreads();
           int tot[9];
 #pragma unroll
-          for (int b = 0; b < 9; ++b) {
-            tot[b] = 0;
-            for (int w = 0; w < kSelWarps; ++w) tot[b] += wc[w * 9 + b];
-          }
-          __syncthreads();
+          for (int b = 0; b < 9; ++b) tot[b] = lead_b[b];
           if (tot[8] < remaining) {
             int above = tot[8], b = 7;
             for (; b > 0; --b) {
@@ -487,12 +485,13 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         const int need_eq = remaining;
         // ---- winners and ties into position bitmaps, then out in ascending position
         const int n_words = (g.e + 31) >> 5;
-        {
+        if (maps_dirty) {                                    // the first selection found them cleared during the gather
           uint4* z4 = reinterpret_cast<uint4*>(map_gt);      // both bitmaps, adjacent, whole 16-byte words
           const int n4 = (p.bitmap_words + ((n_words + 3) & ~3)) >> 2;
           for (int w = tid; w < n4; w += kSelThreads) z4[w] = make_uint4(0u, 0u, 0u, 0u);
+          __syncthreads();
         }
-        __syncthreads();
+        maps_dirty = true;
         for (int i = tid; i < n_cand; i += kSelThreads) {
           const uint2 c = cand[i];
           if (c.y == kNoSelection) continue;
@@ -510,23 +509,44 @@ __global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const Str
         int gt0 = 0, eq0 = 0, gt1 = 0, eq1 = 0;
         for (int w = 2 * tid * gw; w < min((2 * tid + 1) * gw, n_words); ++w) { gt0 += __popc(map_gt[w]); eq0 += __popc(map_eq[w]); }
         for (int w = (2 * tid + 1) * gw; w < min((2 * tid + 2) * gw, n_words); ++w) { gt1 += __popc(map_gt[w]); eq1 += __popc(map_eq[w]); }
-        int tot_gt, tot_eq;
-        const int sg = block_exclusive_scan(gt0 + gt1, wsum, tot_gt);
-        __syncthreads();
-        const int sq = block_exclusive_scan(eq0 + eq1, wsum, tot_eq);
+        // one scan for both counts, 16 bits each (a finishing CTA holds fewer than 2^15 candidates)
+        int tot_packed;
+        const int sp = block_exclusive_scan((gt0 + gt1) | ((eq0 + eq1) << 16), wsum, tot_packed);
+        const int sg = sp & 0xffff, sq = sp >> 16;
         grp_gt[2 * tid] = sg; grp_gt[2 * tid + 1] = sg + gt0;
         grp_eq[2 * tid] = sq; grp_eq[2 * tid + 1] = sq + eq0;
         __syncthreads();
+        if (gshift == 2) {
+          // groups of four words: a group of either bitmap is one 16-byte read
 #pragma unroll 2
-        for (int i = tid; i < n_cand; i += kSelThreads) {
-          const uint2 c = cand[i];
-          if (c.x < T || c.y == kNoSelection) continue;
-          const int w = (int)(c.y >> 5), grp = w >> gshift;
-          const uint32_t below = (1u << (c.y & 31)) - 1u;
-          int g_before = grp_gt[grp] + __popc(map_gt[w] & below), q_before = grp_eq[grp] + __popc(map_eq[w] & below);
-          for (int ww = grp << gshift; ww < w; ++ww) { g_before += __popc(map_gt[ww]); q_before += __popc(map_eq[ww]); }
-          if (c.x > T) idx[g_before + min(q_before, need_eq)] = (int32_t)c.y;
-          else if (q_before < need_eq) idx[g_before + q_before] = (int32_t)c.y;
+          for (int i = tid; i < n_cand; i += kSelThreads) {
+            const uint2 c = cand[i];
+            if (c.x < T || c.y == kNoSelection) continue;
+            const int w = (int)(c.y >> 5), grp = w >> 2, sub = w & 3;
+            const uint32_t below = (1u << (c.y & 31)) - 1u;
+            const uint4 mg = reinterpret_cast<const uint4*>(map_gt)[grp], mq = reinterpret_cast<const uint4*>(map_eq)[grp];
+            // words of the group before mine count whole, mine up to my bit, the rest not at all
+            const uint32_t k0 = sub > 0 ? 0xffffffffu : (sub == 0 ? below : 0u);
+            const uint32_t k1 = sub > 1 ? 0xffffffffu : (sub == 1 ? below : 0u);
+            const uint32_t k2 = sub > 2 ? 0xffffffffu : (sub == 2 ? below : 0u);
+            const uint32_t k3 = sub == 3 ? below : 0u;
+            const int g_before = grp_gt[grp] + __popc(mg.x & k0) + __popc(mg.y & k1) + __popc(mg.z & k2) + __popc(mg.w & k3);
+            const int q_before = grp_eq[grp] + __popc(mq.x & k0) + __popc(mq.y & k1) + __popc(mq.z & k2) + __popc(mq.w & k3);
+            if (c.x > T) idx[g_before + min(q_before, need_eq)] = (int32_t)c.y;
+            else if (q_before < need_eq) idx[g_before + q_before] = (int32_t)c.y;
+          }
+        } else {
+#pragma unroll 2
+          for (int i = tid; i < n_cand; i += kSelThreads) {
+            const uint2 c = cand[i];
+            if (c.x < T || c.y == kNoSelection) continue;
+            const int w = (int)(c.y >> 5), grp = w >> gshift;
+            const uint32_t below = (1u << (c.y & 31)) - 1u;
+            int g_before = grp_gt[grp] + __popc(map_gt[w] & below), q_before = grp_eq[grp] + __popc(map_eq[w] & below);
+            for (int ww = grp << gshift; ww < w; ++ww) { g_before += __popc(map_gt[ww]); q_before += __popc(map_eq[ww]); }
+            if (c.x > T) idx[g_before + min(q_before, need_eq)] = (int32_t)c.y;
+            else if (q_before < need_eq) idx[g_before + q_before] = (int32_t)c.y;
+          }
         }
       }
     } else {
