@@ -716,6 +716,34 @@ def test_topk_structured_score_vectors_exact_and_not_slow(B, W, oracle):
         assert t <= 3.0 * base + 0.02, "%s takes %.3f ms against %.3f ms for random scores" % (key, t, base)
 
 
+def test_topk_short_units_in_one_cta_and_streamed(B, W, oracle):
+    """Units of up to 16381 positions are selected by one CTA each (scores, floor sample, candidates and the
+    finishing step all in shared memory); many hundreds of such units with a workspace are streamed
+    instead.  Both against the oracle: sizes at the one-CTA limit, odd offsets of the units in memory,
+    empty and tiny sequences, a forced tail, structured scores, heavy ties, a second budget."""
+    rng = np.random.default_rng(61)
+    for n in (16381, 16382, 16384, 9001):                     # 16384 (units on 16-byte boundaries) and 16381 (anywhere) are the longest
+        x = (rng.random((1, 2, n)) ** 6).astype(np.float32)
+        run_topk_case(B, W, oracle, x, [0, n], 0, 7, 1024, 0)
+    # sequences at odd offsets (a unit's first score on any 4-byte boundary), one empty, one tiny
+    cu = [0, 16381, 16381, 16384, 27003, 39990]
+    x = (rng.random((2, 3, cu[-1])) ** 5).astype(np.float32)
+    run_topk_case(B, W, oracle, x, cu, 0, 7, 1500, 0)
+    run_topk_case(B, W, oracle, x, cu, 0, 7, 1500, 32)
+    run_vert_case(B, oracle, x, cu, 7, 1024, 32, 2048)
+    for name, fn in STRUCTURED.items():
+        y = np.stack([fn(rng, 12000) for _ in range(3)])[None].astype(np.float32)
+        run_topk_case(B, W, oracle, y, [0, 12000], 0, 7, 2000, 0)
+        run_vert_case(B, oracle, y, [0, 5000, 12000], 7, 300, 16, 700)
+    y = np.zeros((1, 2, 8000), np.float32)                        # every key equal: the generic selection
+    run_topk_case(B, W, oracle, y, [0, 8000], 0, 7, 1000, 0)
+    # 640 units of 3000 with a workspace: more units than the one-CTA kernel is given, so they are streamed
+    z = (rng.random((40, 16, 3000)) ** 4).astype(np.float32)
+    z[:, :, 100:140] = 0.75                                          # a run of ties around the threshold of some units
+    run_topk_case(B, W, oracle, z, [0, 3000], 0, 7, 256, 0)
+    run_vert_case(B, oracle, z, [0, 1000, 3000], 7, 128, 8, 150)
+
+
 def test_topk_unit_too_long_for_a_cluster_takes_the_generic_path(B, W, oracle):
     rng = np.random.default_rng(41)
     n = 2_000_003
