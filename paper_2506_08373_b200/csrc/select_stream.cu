@@ -525,7 +525,7 @@ __host__ __device__ inline size_t stream_finish_bytes(int bitmap_words, int held
   return (size_t)kStreamBins * 4 + (size_t)held_cap * 8 + (maps > generic ? maps : generic);
 }
 
-__global__ void __launch_bounds__(kSelThreads, 2) stream_finish_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(kSelThreads, 3) stream_finish_kernel(const StreamParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __shared__ int wsum[32];
   __shared__ int out2[4];
