@@ -225,13 +225,13 @@ __device__ __forceinline__ uint32_t sweep_steps(const SweepItem& t, const float*
       const float4* at = base4 + st * 32 + lane;
       const float4 pv = at[-1], cv = at[0], nv = at[1];
       const float x[10] = {pv.y, pv.z, pv.w, cv.x, cv.y, cv.z, cv.w, nv.x, nv.y, nv.z};
-      float t3[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) t3[i] = fmax3(x[i], x[i + 1], x[i + 2]);
+      // the four windows share x[3..6]; neighbouring windows share a pair on either side
+      const float mid = fmax3(x[3], x[4], fmaxf(x[5], x[6])), l12 = fmaxf(x[1], x[2]), r78 = fmaxf(x[7], x[8]);
+      const float v[4] = {fmax3(mid, x[0], l12), fmax3(mid, l12, x[7]), fmax3(mid, x[2], r78), fmax3(mid, r78, x[9])};
       const int pp0 = t.x0 + st * 128 + lane * 4 - t.mis;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        bool c = !(fmax3(t3[u], t3[u + 3], x[u + 6]) < floor_f);
+        bool c = !(v[u] < floor_f);
         if (EDGE) c = c && pp0 + u >= 0 && pp0 + u < t.g.e;
         if (c) mask |= 1u << (4 * k + u);
       }
@@ -700,9 +700,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) unit_select_kernel(const Strea
             const float4* a4 = base4 + st * 32 + lane;
             const float4 pv = a4[-1], cv = a4[0], nv = a4[1];
             const float x[10] = {pv.y, pv.z, pv.w, cv.x, cv.y, cv.z, cv.w, nv.x, nv.y, nv.z};
-            const float mid = fmax3(x[3], x[4], fmaxf(x[5], x[6]));                  // in all four windows
-            const float v[4] = {fmax3(mid, x[0], fmaxf(x[1], x[2])), fmax3(mid, x[1], fmaxf(x[2], x[7])),
-                                fmax3(mid, x[2], fmaxf(x[7], x[8])), fmax3(mid, x[7], fmaxf(x[8], x[9]))};
+            const float mid = fmax3(x[3], x[4], fmaxf(x[5], x[6])), l12 = fmaxf(x[1], x[2]), r78 = fmaxf(x[7], x[8]);
+            const float v[4] = {fmax3(mid, x[0], l12), fmax3(mid, l12, x[7]), fmax3(mid, x[2], r78), fmax3(mid, r78, x[9])};
             const int j0 = st * 128 + lane * 4 - t.mis;                              // position of my first slot
 #pragma unroll
             for (int u = 0; u < 4; ++u)
