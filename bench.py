@@ -44,8 +44,11 @@ NCU_TRAFFIC = {
     # workload index -> {kernel group: (bytes per layer, source files, hash of those sources)}
     # profiles/score_kernel_c2.md (2 layers) and profiles/select_and_gather_c2.md (8 layers)
     2: {"score": ((542.008064e6 + 7.79392e6 + 550.035456e6 + 11.079168e6) / 2, ["score.cu"], "d44fc0da3556a83b"),
-        "select": ((8.40576e6 + 33.587712e6 + 0.007168e6 + 3.372544e6) / 8, ["select_stream.cu", "select_common.cuh"], "1c90281812721d22"),
-        "gather": ((67.677696e6 + 13.709824e6) / 8, ["compact.cu"], "4de11f4bd31ee049")},
+        "select": ((8.407296e6 + 33.585152e6 + 0.004864e6 + 3.372288e6) / 8, ["select_stream.cu", "select_common.cuh"], "85dd21fd6eafcc5a"),
+        "gather": ((67.679488e6 + 13.955328e6) / 8, ["compact.cu"], "4de11f4bd31ee049")},
+    # profiles/select_and_gather_c2.md, the capture of all 32 layers of workload 1 (unit_select_kernel, compact_bulk_kernel)
+    1: {"select": (16.861952e6 / 32, ["select_stream.cu", "select_common.cuh"], "85dd21fd6eafcc5a"),
+        "gather": ((135.294976e6 + 75.415808e6) / 32, ["compact.cu"], "4de11f4bd31ee049")},
 }
 
 
@@ -246,8 +249,15 @@ class State:
             # what the path produces: the index lists and the compacted cache
             self.results = [self.idx, self.cnt, self.k_out, self.v_out]
         # kernels of the library per step: two scoring passes + merge; keep set: reduce + cluster select;
-        # else sample floor + sweep + finish, and the gather
-        self.launches_per_step = 3 + ((3 if w.paper_specpc else 2) if self.specpc else 4)
+        # else the selection (sample floor + sweep + finish; one kernel for up to 592 units of up to 16384
+        # positions, and for a budget above a sixth of the sequence) and the gather
+        max_len = w.len_hi if w.n_seq > 1 else w.n_in
+        n_units = w.n_seq * self.L * w.n_kv_heads
+        self.select_kernels = ("sample_floor + stream_sweep + stream_finish" if w.c_max * 6 <= max_len and
+                               (max_len + 3 > 16384 + (3 if w.n_seq == 1 else 0) or n_units > 592) else
+                               "unit_select" if w.c_max * 6 <= max_len else "cluster_select")
+        self.launches_per_step = 3 + ((3 if w.paper_specpc else 2) if self.specpc else
+                                      (3 if self.select_kernels.startswith("sample") else 1) + 1)
 
     def step(self, events=None, v_src=None):
         B, w = self.B, self.w
@@ -477,7 +487,7 @@ def main(argv=None):
                 "algorithmic_bytes": work["score_hbm_bytes"], "traffic": ncu_traffic(args.config, "score", st.L)}
     hbm_bytes = work["select_bytes"] + work["gather_bytes"]
     gbs = hbm_bytes / ((t_select + t_gather) * 1e-3) / 1e9
-    roofline_hbm = {"bound": "hbm", "kernel": ("sample_floor + stream_sweep + stream_finish + compact_bulk" if not st.specpc
+    roofline_hbm = {"bound": "hbm", "kernel": (st.select_kernels + " + compact_bulk" if not st.specpc
                                                  else "token_reduce + cluster_select"),
                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                     "peak_source": peak_src + " (copy)", "ms_select": t_select, "ms_gather": t_gather,
