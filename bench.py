@@ -44,10 +44,10 @@ NCU_TRAFFIC = {
     # workload index -> {kernel group: (bytes per layer, source files, hash of those sources)}
     # profiles/score_kernel_c2.md (2 layers) and profiles/select_and_gather_c2.md (8 layers)
     2: {"score": ((542.008064e6 + 7.79392e6 + 550.035456e6 + 11.079168e6) / 2, ["score.cu"], "d44fc0da3556a83b"),
-        "select": ((8.407296e6 + 33.585152e6 + 0.004864e6 + 3.372288e6) / 8, ["select_stream.cu", "select_common.cuh"], "85dd21fd6eafcc5a"),
+        "select": ((8.407296e6 + 33.585152e6 + 0.004864e6 + 3.372288e6) / 8, ["select_stream.cu", "select_common.cuh"], "44e0bb49c4dfc6e9"),
         "gather": ((67.679488e6 + 13.955328e6) / 8, ["compact.cu"], "4de11f4bd31ee049")},
     # profiles/select_and_gather_c2.md, the capture of all 32 layers of workload 1 (unit_select_kernel, compact_bulk_kernel)
-    1: {"select": (16.861952e6 / 32, ["select_stream.cu", "select_common.cuh"], "85dd21fd6eafcc5a"),
+    1: {"select": (16.861952e6 / 32, ["select_stream.cu", "select_common.cuh"], "44e0bb49c4dfc6e9"),
         "gather": ((135.294976e6 + 75.415808e6) / 32, ["compact.cu"], "4de11f4bd31ee049")},
 }
 

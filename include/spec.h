@@ -147,8 +147,9 @@ int32_t spec_score(const spec_problem* problem, const void* q, const void* k, co
  *  count_out  optional [n_seq, n_layers, n_kv_heads] int32 number of valid entries
  * Requires 1 <= pool_k <= 255, 0 <= n_forced_tail <= c_max, c_max >= 1.
  * workspace is optional (NULL, 0): the lists are the same either way.  With a workspace of
- * spec_workspace_bytes() the default pooling (SPEC_POOL_MAX, pool_k = 7) takes its fastest path,
- * which parks candidate positions there.
+ * spec_workspace_bytes() the default pooling (SPEC_POOL_MAX, pool_k = 7) takes its fastest path
+ * for sequences beyond 16384 positions, which parks candidate positions there; shorter
+ * sequences with that pooling are selected in shared memory alone and need none.
  */
 int32_t spec_pool_topk(const spec_problem* problem, const float* scores, int32_t pool, int32_t pool_k,
                        int32_t c_max, int32_t n_forced_tail, int32_t* idx_out, int32_t* count_out,

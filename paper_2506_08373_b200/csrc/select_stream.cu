@@ -21,6 +21,9 @@
 // If the floor was too high or too low for the candidate array (fewer candidates than the budget,
 // or more than fit: only with massively tied scores), the finishing CTA falls back to the generic
 // selection that recomputes pooled keys from global memory.  The result is exact in every case.
+//
+// Units of up to 16384 positions, a few to an SM, skip the workspace and the three launches:
+// unit_select_kernel stages a unit in shared memory and does the same three steps in one CTA.
 #include "select_common.cuh"
 
 #include <algorithm>
